@@ -1,0 +1,196 @@
+/*
+ * rvq.h -- C ABI of the B200 residual-vector-quantization KV-cache library.
+ *
+ * The library implements the data-parallel part of "Residual vector
+ * quantization for KV cache compression in large language model":
+ *   - encode  (Section 2.2 + Algorithm 1): scale a head vector by its standard
+ *     deviation, split its channels into groups (Section 3.1: contiguous, or
+ *     channels d/d^ apart), run R greedy stages of nearest-code search and
+ *     residual subtraction against one shared set of R codebooks;
+ *   - decode  (Section 2.2, last sentence): sum the R chosen codes per group,
+ *     un-group, multiply by the stored standard deviation (Section 3.2: kept in
+ *     half precision);
+ *   - EMA codebook update (Section 3: exponential moving average, decay 0.99).
+ *
+ * Conventions shared by every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless its
+ *     comment says "host".  The library never allocates, frees or keeps a
+ *     pointer after the call returns.  Work is enqueued on `stream` and the
+ *     call returns without synchronising.
+ *   - n     number of head vectors (tokens x heads); dim channels each.
+ *     G = dim / group_dim groups per vector, R = depth, K = codebook_size.
+ *   - codebooks: float32 [R][K][group_dim], row-major, 16-byte aligned.
+ *   - x / x_out: n rows of `dim` contiguous elements of `x_dtype`; row v starts
+ *     at element v * row_stride.  16-byte aligned base, row_stride * element
+ *     size a multiple of 16 bytes.
+ *   - codes: code_bits == 16: uint16 [n][G][R].  Otherwise code_bits must be
+ *     ceil(log2 K) and each head vector is a little-endian bit stream, code
+ *     number g*R+r at bit offset code_bits*(g*R+r), least significant bit
+ *     first, padded to a multiple of 4 bytes (rvq_code_bytes()).
+ *   - std: uint16 [n] holding IEEE binary16 bit patterns.
+ *   - Return value: RVQ_OK or a negative rvq_error.  Argument errors are
+ *     detected on the host before anything is launched.  Conditions found on
+ *     the device are counted in the optional `rvq_status` block (device memory,
+ *     zeroed by the caller, read by the caller after the stream has drained).
+ */
+#ifndef RVQ_H
+#define RVQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { RVQ_F32 = 0, RVQ_BF16 = 1, RVQ_F16 = 2 } rvq_dtype;
+typedef enum { RVQ_GROUP_CONTIGUOUS = 0, RVQ_GROUP_STRIDED = 1 } rvq_layout;
+
+typedef enum {
+    RVQ_OK = 0,
+    RVQ_ERR_BADARG = -1,       /* null pointer, negative size, value out of range   */
+    RVQ_ERR_ALIGN = -2,        /* pointer or stride not 16-byte aligned              */
+    RVQ_ERR_UNSUPPORTED = -3,  /* shape outside what the kernels handle              */
+    RVQ_ERR_WORKSPACE = -4,    /* workspace smaller than rvq_workspace_bytes()       */
+    RVQ_ERR_LAUNCH = -5,       /* the CUDA runtime refused a launch or a copy        */
+    RVQ_ERR_DEVICE = -6        /* not an sm_100 device, or no device                 */
+} rvq_error;
+
+/* Shape of one quantizer (Section 3: default dim 128, group_dim 32, depth 8,
+ * codebook_size 2048). */
+typedef struct rvq_config {
+    int32_t dim;            /* channels per head vector, <= 1024, multiple of group_dim */
+    int32_t group_dim;      /* d^: 8, 16, 32 or 64                                      */
+    int32_t layout;         /* rvq_layout (Section 3.1)                                 */
+    int32_t depth;          /* R, 1..16 (the paper's K)                                 */
+    int32_t codebook_size;  /* K, 2..65536 (the paper's |C_i|)                          */
+    int32_t code_bits;      /* 16, or ceil(log2 K) for the packed form (Section 3.2)    */
+    int32_t x_dtype;        /* rvq_dtype of vectors in (encode, EMA) and out (decode)   */
+    int32_t std_ddof;       /* 0: population deviation (default); 1: sample deviation   */
+} rvq_config;
+
+/* Device-side counters.  Zero the block before a call, read it after the
+ * stream has drained.  Counters accumulate over calls. */
+typedef struct rvq_status {
+    uint32_t degenerate_vectors;  /* zero or non-finite deviation: codes 0, std 0         */
+    uint32_t std_out_of_half;     /* deviation overflowed / underflowed binary16          */
+    uint32_t rescored_rows;       /* (row, stage) pairs sent through the exact re-scoring */
+    uint32_t exhaustive_rows;     /* (row, stage) pairs that fell back to a full scan     */
+    uint32_t wait_timeouts;       /* bounded waits that gave up (result invalid if != 0)  */
+    uint32_t bad_codes;           /* decode / EMA met a code >= K (treated as code 0)     */
+    uint32_t reserved[2];
+} rvq_status;
+
+/* Text for a return value (host pointer to a static string). */
+const char *rvq_status_string(int code);
+
+/* Library version, major * 1000 + minor. */
+int rvq_version(void);
+
+/* Diagnostic: number of kernels this library has launched in this process so
+ * far (the only process-wide state it keeps). */
+uint64_t rvq_launch_count(void);
+
+/* Bytes of one head vector's codes in the configured storage form
+ * (Section 3.2: G*R indices of code_bits bits).  0 on a bad config. */
+size_t rvq_code_bytes(const rvq_config *cfg /* host */);
+
+/* Size of the prepared-codebook block for this shape. 0 on a bad config. */
+size_t rvq_prepared_bytes(const rvq_config *cfg /* host */);
+
+/*
+ * Derive, from the float32 codebooks, everything the kernels read instead of
+ * them: half-precision copies in the tensor-core operand layout with their
+ * squared norms and rounding-error bounds (Algorithm 1's argmin, expanded as
+ * ||e||^2 - 2 z.e), and the fixed-point channel-sliced tables of the decoder.
+ * `prepared` (device, 256-byte aligned, rvq_prepared_bytes() bytes) is
+ * overwritten.  Must be called again after every change of the codebooks,
+ * on the same stream or after synchronising.
+ */
+int rvq_prepare_codebooks(const rvq_config *cfg /* host */, const float *codebooks,
+                          void *prepared, void *stream /* cudaStream_t */);
+
+/* Scratch bytes rvq_encode / rvq_ema_stats / rvq_ema_update need for n head vectors. */
+size_t rvq_workspace_bytes(const rvq_config *cfg /* host */, int64_t n);
+
+/*
+ * Encode (Section 2.2, Algorithm 1).  For each of the n head vectors: deviation
+ * s over its dim channels (x is not centred), z = x / s, grouping, then for
+ * r = 0..R-1: j = argmin_j ||z_r - C_r[j]||^2 under exact squared Euclidean
+ * distance (lowest index on ties), z_{r+1} = z_r - C_r[j].
+ *   x            in   n rows of x_dtype
+ *   codebooks    in   float32 [R][K][group_dim]
+ *   prepared     in   block written by rvq_prepare_codebooks for these codebooks
+ *   codes        out  see "codes" above; rvq_code_bytes() * n bytes
+ *   std_f16      out  binary16 rounding of s (the scaling itself uses s unrounded)
+ *   workspace         rvq_workspace_bytes(cfg, n) bytes, 256-byte aligned; may be
+ *                     NULL when that size is 0
+ *   status            optional counters (may be NULL)
+ * A vector whose deviation is zero or not finite gets codes 0 and std 0.
+ */
+int rvq_encode(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
+               const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+               void *workspace, size_t workspace_bytes, rvq_status *status,
+               void *stream /* cudaStream_t */);
+
+/*
+ * Decode (Section 2.2, last sentence; Section 3.2).  For every head vector and
+ * channel c = channel(g, i): x_out[c] = std * sum_r C_r[code[g][r]][i], summed
+ * in float32 in stage order and rounded once to x_dtype.
+ *   codes, std_f16  in   as produced by rvq_encode
+ *   x_out           out  n rows of x_dtype, row v at element v * out_row_stride
+ * A code >= K is read as code 0 and counted in status->bad_codes.
+ */
+int rvq_decode(const rvq_config *cfg /* host */, const void *codes, const uint16_t *std_f16,
+               int64_t n, const float *codebooks, const void *prepared, void *x_out,
+               int64_t out_row_stride, rvq_status *status, void *stream /* cudaStream_t */);
+
+/*
+ * One EMA codebook update (Section 3: "update them using exponential moving
+ * average with a decay factor of 0.99"; Section 2.1: EMA in place of the
+ * codebook loss).  With n_r[j] the number of group rows whose stage-r code is j
+ * and m_r[j] the sum of their stage-r inputs z_r (scaled space, rebuilt from x,
+ * the codes and the codebooks passed in):
+ *   N <- decay N + (1 - decay) n ;   M <- decay M + (1 - decay) m ;
+ *   N^_j = (N_j + eps) * sum_j N / (sum_j N + K eps) ;   C_r[j] <- M_r[j] / N^_j.
+ *   x, codes     in      the vectors and the codes rvq_encode chose for them
+ *                        with these same codebooks
+ *   codebooks    in/out  float32 [R][K][group_dim]
+ *   ema_count    in/out  float32 [R][K]              (N)
+ *   ema_sum      in/out  float32 [R][K][group_dim]   (M)
+ *   batch_count  out     optional float32 [R][K]: n of this call (may be NULL)
+ *   workspace            rvq_workspace_bytes(cfg, n) bytes, 256-byte aligned
+ * The caller must call rvq_prepare_codebooks again before the next encode or
+ * decode.  Equivalent to rvq_ema_stats followed by rvq_ema_apply.
+ */
+int rvq_ema_update(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
+                   const void *codes, float *codebooks, float *ema_count, float *ema_sum,
+                   float *batch_count, float decay, float eps, void *workspace,
+                   size_t workspace_bytes, rvq_status *status, void *stream /* cudaStream_t */);
+
+/*
+ * The two halves of rvq_ema_update, for data-parallel codebook learning: every
+ * device computes the statistics of its own vectors, the caller sums
+ * batch_count and batch_sum over devices (the counts and sums of Section 3's
+ * moving average are plain sums over vectors), then every device applies the
+ * same update.
+ *   batch_count  out  float32 [R][K]             n_r[j] of these n vectors
+ *                     (exact while a bin holds fewer than 2^24 rows)
+ *   batch_sum    out  float32 [R][K][group_dim]  m_r[j]; 16-byte aligned
+ * Both are overwritten.  Workspace as for rvq_ema_update.
+ */
+int rvq_ema_stats(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
+                  const void *codes, const float *codebooks, float *batch_count, float *batch_sum,
+                  void *workspace, size_t workspace_bytes, rvq_status *status,
+                  void *stream /* cudaStream_t */);
+
+/* N, M and the codebooks updated in place from the given batch statistics
+ * (formulas under rvq_ema_update). */
+int rvq_ema_apply(const rvq_config *cfg /* host */, const float *batch_count,
+                  const float *batch_sum, float *codebooks, float *ema_count, float *ema_sum,
+                  float decay, float eps, void *stream /* cudaStream_t */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RVQ_H */

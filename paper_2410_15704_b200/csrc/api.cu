@@ -1,0 +1,193 @@
+// extern "C" boundary of the RVQ library: argument checks on the host, then
+// dispatch to the kernels.  No allocation, no synchronisation, no global state.
+#include "common.cuh"
+
+#include <atomic>
+
+namespace rvq {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+static int ceil_log2(int k)
+{
+    int b = 0;
+    while ((1 << b) < k) ++b;
+    return b < 1 ? 1 : b;
+}
+
+int make_shape(const rvq_config *c, Shape *s)
+{
+    if (!c) return RVQ_ERR_BADARG;
+    if (c->group_dim != 8 && c->group_dim != 16 && c->group_dim != 32 && c->group_dim != 64)
+        return RVQ_ERR_UNSUPPORTED;
+    if (c->dim < c->group_dim || c->dim > 1024 || c->dim % c->group_dim) return RVQ_ERR_BADARG;
+    if (c->layout != RVQ_GROUP_CONTIGUOUS && c->layout != RVQ_GROUP_STRIDED) return RVQ_ERR_BADARG;
+    if (c->depth < 1 || c->depth > 16) return RVQ_ERR_BADARG;
+    if (c->codebook_size < 2 || c->codebook_size > 65536) return RVQ_ERR_BADARG;
+    if (c->code_bits != 16 && c->code_bits != ceil_log2(c->codebook_size)) return RVQ_ERR_BADARG;
+    if (c->x_dtype < RVQ_F32 || c->x_dtype > RVQ_F16) return RVQ_ERR_BADARG;
+    if (c->std_ddof != 0 && c->std_ddof != 1) return RVQ_ERR_BADARG;
+    s->dim = c->dim; s->gd = c->group_dim; s->G = c->dim / c->group_dim; s->layout = c->layout;
+    s->R = c->depth; s->K = c->codebook_size; s->bits = c->code_bits; s->dtype = c->x_dtype;
+    s->ddof = c->std_ddof;
+    if (s->G > 128 || s->dim - s->ddof <= 0) return RVQ_ERR_UNSUPPORTED;
+    s->per_vector = s->G * s->R;
+    s->code_bytes = (s->per_vector * s->bits + 31) / 32 * 4;
+    s->elem_bytes = c->x_dtype == RVQ_F32 ? 4 : 2;
+    return RVQ_OK;
+}
+
+static int check_rows(const Shape &s, const void *p, int64_t n, int64_t stride)
+{
+    if (n < 0 || stride < s.dim) return RVQ_ERR_BADARG;
+    if (n > 0 && !p) return RVQ_ERR_BADARG;
+    if (!aligned16(p) || (stride * s.elem_bytes) % 16) return RVQ_ERR_ALIGN;
+    return RVQ_OK;
+}
+
+}  // namespace rvq
+
+using namespace rvq;
+
+extern "C" {
+
+const char *rvq_status_string(int code)
+{
+    switch (code) {
+    case RVQ_OK: return "ok";
+    case RVQ_ERR_BADARG: return "bad argument";
+    case RVQ_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+    case RVQ_ERR_UNSUPPORTED: return "unsupported shape";
+    case RVQ_ERR_WORKSPACE: return "workspace too small";
+    case RVQ_ERR_LAUNCH: return "CUDA launch failed";
+    case RVQ_ERR_DEVICE: return "no sm_100 device";
+    default: return "unknown error";
+    }
+}
+
+int rvq_version(void) { return 1000; }
+
+uint64_t rvq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t rvq_code_bytes(const rvq_config *cfg)
+{
+    Shape s;
+    return make_shape(cfg, &s) == RVQ_OK ? (size_t)s.code_bytes : 0;
+}
+
+size_t rvq_prepared_bytes(const rvq_config *cfg)
+{
+    Shape s;
+    return make_shape(cfg, &s) == RVQ_OK ? prepared_bytes(s) : 0;
+}
+
+int rvq_prepare_codebooks(const rvq_config *cfg, const float *codebooks, void *prepared, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if (!codebooks || !prepared) return RVQ_ERR_BADARG;
+    if (!aligned16(codebooks) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    return launch_prepare(s, codebooks, prepared, (cudaStream_t)stream);
+}
+
+size_t rvq_workspace_bytes(const rvq_config *cfg, int64_t n)
+{
+    Shape s;
+    (void)n;
+    return make_shape(cfg, &s) == RVQ_OK ? ema_workspace_bytes(s) : 0;
+}
+
+int rvq_encode(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+               const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+               void *workspace, size_t workspace_bytes, rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if ((rc = check_rows(s, x, n, x_row_stride)) != RVQ_OK) return rc;
+    if (!codebooks || !prepared || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
+    if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    (void)workspace; (void)workspace_bytes;
+    return launch_encode_scalar(s, x, n, x_row_stride, codebooks, codes, std_f16, status, (cudaStream_t)stream);
+}
+
+int rvq_decode(const rvq_config *cfg, const void *codes, const uint16_t *std_f16, int64_t n,
+               const float *codebooks, const void *prepared, void *x_out, int64_t out_row_stride,
+               rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if ((rc = check_rows(s, x_out, n, out_row_stride)) != RVQ_OK) return rc;
+    if (!codebooks || !prepared || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
+    if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    return launch_decode_gather(s, codes, std_f16, n, codebooks, x_out, out_row_stride, status, (cudaStream_t)stream);
+}
+
+static int check_ema_common(const Shape &s, const void *x, int64_t n, int64_t stride, const void *codes,
+                            const float *codebooks)
+{
+    int rc = check_rows(s, x, n, stride);
+    if (rc != RVQ_OK) return rc;
+    if (!codebooks || (n > 0 && !codes)) return RVQ_ERR_BADARG;
+    if (!aligned16(codebooks) || !aligned16(codes)) return RVQ_ERR_ALIGN;
+    return RVQ_OK;
+}
+
+int rvq_ema_stats(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                  const void *codes, const float *codebooks, float *batch_count, float *batch_sum,
+                  void *workspace, size_t workspace_bytes, rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if ((rc = check_ema_common(s, x, n, x_row_stride, codes, codebooks)) != RVQ_OK) return rc;
+    if (!batch_count || !batch_sum || !workspace) return RVQ_ERR_BADARG;
+    if (!aligned16(batch_sum) || !aligned256(workspace)) return RVQ_ERR_ALIGN;
+    if (workspace_bytes < ema_stats_scratch_bytes(s)) return RVQ_ERR_WORKSPACE;
+    return launch_ema_stats(s, x, n, x_row_stride, codes, codebooks, batch_count, batch_sum, workspace,
+                            status, (cudaStream_t)stream);
+}
+
+int rvq_ema_apply(const rvq_config *cfg, const float *batch_count, const float *batch_sum,
+                  float *codebooks, float *ema_count, float *ema_sum, float decay, float eps,
+                  void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if (!batch_count || !batch_sum || !codebooks || !ema_count || !ema_sum) return RVQ_ERR_BADARG;
+    if (!(decay >= 0.0f && decay <= 1.0f) || !(eps >= 0.0f)) return RVQ_ERR_BADARG;
+    return launch_ema_apply(s, batch_count, batch_sum, codebooks, ema_count, ema_sum, decay, eps,
+                            (cudaStream_t)stream);
+}
+
+int rvq_ema_update(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                   const void *codes, float *codebooks, float *ema_count, float *ema_sum,
+                   float *batch_count, float decay, float eps, void *workspace,
+                   size_t workspace_bytes, rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if ((rc = check_ema_common(s, x, n, x_row_stride, codes, codebooks)) != RVQ_OK) return rc;
+    if (!ema_count || !ema_sum || !workspace) return RVQ_ERR_BADARG;
+    if (!(decay >= 0.0f && decay <= 1.0f) || !(eps >= 0.0f)) return RVQ_ERR_BADARG;
+    if (!aligned16(ema_sum) || !aligned256(workspace)) return RVQ_ERR_ALIGN;
+    if (workspace_bytes < ema_workspace_bytes(s)) return RVQ_ERR_WORKSPACE;
+    uint8_t *ws = reinterpret_cast<uint8_t *>(workspace);
+    float *bc = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s));
+    float *bs = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s) +
+                                          ((size_t)s.R * s.K * sizeof(float) + 255) / 256 * 256);
+    rc = launch_ema_stats(s, x, n, x_row_stride, codes, codebooks, bc, bs, workspace, status, (cudaStream_t)stream);
+    if (rc != RVQ_OK) return rc;
+    if (batch_count &&
+        cudaMemcpyAsync(batch_count, bc, (size_t)s.R * s.K * sizeof(float), cudaMemcpyDeviceToDevice,
+                        (cudaStream_t)stream) != cudaSuccess)
+        return RVQ_ERR_LAUNCH;
+    return launch_ema_apply(s, bc, bs, codebooks, ema_count, ema_sum, decay, eps, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,149 @@
+// EMA codebook update (Section 3; Section 2.1).  Two kernels: per-code counts
+// and sums of the stage inputs, then the decayed, Laplace-smoothed
+// normalisation.
+#include "common.cuh"
+
+namespace rvq {
+
+static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
+
+// rvq_ema_stats scratch: integer counts, uint32 [R][K].
+size_t ema_stats_scratch_bytes(const Shape &s) { return round256((size_t)s.R * s.K * sizeof(uint32_t)); }
+
+// rvq_ema_update scratch: the above, then batch counts (float [R][K]) and
+// batch sums (float [R][K][gd]).
+size_t ema_workspace_bytes(const Shape &s)
+{
+    return ema_stats_scratch_bytes(s) + round256((size_t)s.R * s.K * sizeof(float)) +
+           (size_t)s.R * s.K * s.gd * sizeof(float);
+}
+
+// One thread per group row: rebuild z_r stage by stage from x, the deviation
+// and the codes, and add it to the bin of its stage-r code.
+template <int GD>
+__global__ void __launch_bounds__(128)
+ema_stats_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t stride,
+                 const void *__restrict__ codes, const float *__restrict__ cb,
+                 uint32_t *__restrict__ cnt, float *__restrict__ sum, rvq_status *st, int vpb)
+{
+    extern __shared__ __align__(16) float smem[];
+    float *xs = smem;
+    float *part = xs + vpb * s.dim;
+    const int tid = threadIdx.x;
+    const int v_local = tid / s.G, g = tid - v_local * s.G;
+    const int64_t v0 = (int64_t)blockIdx.x * vpb;
+    const int64_t gv = v0 + v_local;
+
+    load_tile(xs, x, v0, n, stride, vpb, s.dim, s.dtype);
+    __syncthreads();
+    float z[GD];
+#pragma unroll
+    for (int i = 0; i < GD; ++i) z[i] = xs[v_local * s.dim + channel_of(s.layout, s.G, GD, g, i)];
+    const float dev = block_deviation<GD>(z, part, v_local, s.G, s.dim, s.ddof);
+    const bool deg = deviation_is_degenerate(dev);
+    if (gv >= n) return;
+#pragma unroll
+    for (int i = 0; i < GD; ++i) z[i] = deg ? 0.0f : z[i] / dev;
+
+    const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + gv * s.code_bytes;
+    for (int r = 0; r < s.R; ++r) {
+        uint32_t j = read_code(vec, g * s.R + r, s.bits, s.code_bytes);
+        if (j >= (uint32_t)s.K) { j = 0; if (st) atomicAdd(&st->bad_codes, 1u); }
+        const size_t bin = (size_t)r * s.K + j;
+        atomicAdd(cnt + bin, 1u);
+        float4 *m = reinterpret_cast<float4 *>(sum + bin * GD);
+        const float4 *e = reinterpret_cast<const float4 *>(cb + bin * GD);
+#pragma unroll
+        for (int q = 0; q < GD / 4; ++q) {
+            atomicAdd(m + q, make_float4(z[4 * q], z[4 * q + 1], z[4 * q + 2], z[4 * q + 3]));
+            float4 ev = __ldg(e + q);
+            z[4 * q] -= ev.x; z[4 * q + 1] -= ev.y; z[4 * q + 2] -= ev.z; z[4 * q + 3] -= ev.w;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+counts_to_float_kernel(const uint32_t *__restrict__ cnt, float *__restrict__ out, int total)
+{
+    int t = blockIdx.x * 256 + threadIdx.x;
+    if (t < total) out[t] = (float)cnt[t];
+}
+
+// One block per stage: N <- decay N + (1-decay) n, total = sum_j N, then
+// M <- decay M + (1-decay) m and C = M / ((N + eps) total / (total + K eps)).
+__global__ void __launch_bounds__(256)
+ema_apply_kernel(Shape s, const float *__restrict__ cnt, const float *__restrict__ sum,
+                 float *__restrict__ cb, float *__restrict__ ema_count,
+                 float *__restrict__ ema_sum, float decay, float eps)
+{
+    __shared__ float red[256];
+    const int r = blockIdx.x, tid = threadIdx.x;
+    float local = 0.0f;
+    for (int j = tid; j < s.K; j += 256) {
+        const size_t p = (size_t)r * s.K + j;
+        const float nn = decay * ema_count[p] + (1.0f - decay) * cnt[p];
+        ema_count[p] = nn;
+        local += nn;
+    }
+    red[tid] = local;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (tid < w) red[tid] += red[tid + w];
+        __syncthreads();
+    }
+    const float tot = red[0];
+    const float scale = tot / (tot + (float)s.K * eps);
+    for (int t = tid; t < s.K * s.gd; t += 256) {
+        const size_t p = (size_t)r * s.K * s.gd + t;
+        const int j = t / s.gd;
+        const float mm = decay * ema_sum[p] + (1.0f - decay) * sum[p];
+        ema_sum[p] = mm;
+        cb[p] = mm / ((ema_count[(size_t)r * s.K + j] + eps) * scale);
+    }
+}
+
+template <int GD>
+static int stats_gd(const Shape &s, const void *x, int64_t n, int64_t stride, const void *codes,
+                    const float *cb, uint32_t *cnt, float *sum, rvq_status *st, cudaStream_t stream)
+{
+    const int vpb = 128 / s.G > 0 ? 128 / s.G : 1;
+    const int threads = vpb * s.G;
+    const size_t smem = sizeof(float) * ((size_t)vpb * s.dim + threads);
+    const int64_t blocks = (n + vpb - 1) / vpb;
+    if (blocks > 0x7FFFFFFF) return RVQ_ERR_UNSUPPORTED;
+    ema_stats_kernel<GD><<<(unsigned)blocks, threads, smem, stream>>>(s, x, n, stride, codes, cb, cnt, sum, st, vpb);
+    return check_launch();
+}
+
+int launch_ema_stats(const Shape &s, const void *x, int64_t n, int64_t stride, const void *codes,
+                     const float *cb, float *batch_count, float *batch_sum, void *workspace,
+                     rvq_status *st, cudaStream_t stream)
+{
+    uint32_t *cnt = reinterpret_cast<uint32_t *>(workspace);
+    const int bins = s.R * s.K;
+    if (cudaMemsetAsync(cnt, 0, (size_t)bins * sizeof(uint32_t), stream) != cudaSuccess ||
+        cudaMemsetAsync(batch_sum, 0, (size_t)bins * s.gd * sizeof(float), stream) != cudaSuccess)
+        return RVQ_ERR_LAUNCH;
+    int rc = RVQ_OK;
+    if (n > 0) {
+        switch (s.gd) {
+        case 8: rc = stats_gd<8>(s, x, n, stride, codes, cb, cnt, batch_sum, st, stream); break;
+        case 16: rc = stats_gd<16>(s, x, n, stride, codes, cb, cnt, batch_sum, st, stream); break;
+        case 32: rc = stats_gd<32>(s, x, n, stride, codes, cb, cnt, batch_sum, st, stream); break;
+        case 64: rc = stats_gd<64>(s, x, n, stride, codes, cb, cnt, batch_sum, st, stream); break;
+        default: rc = RVQ_ERR_UNSUPPORTED;
+        }
+    }
+    if (rc != RVQ_OK) return rc;
+    counts_to_float_kernel<<<(bins + 255) / 256, 256, 0, stream>>>(cnt, batch_count, bins);
+    return check_launch();
+}
+
+int launch_ema_apply(const Shape &s, const float *batch_count, const float *batch_sum, float *cb,
+                     float *ema_count, float *ema_sum, float decay, float eps, cudaStream_t stream)
+{
+    ema_apply_kernel<<<s.R, 256, 0, stream>>>(s, batch_count, batch_sum, cb, ema_count, ema_sum, decay, eps);
+    return check_launch();
+}
+
+}  // namespace rvq

@@ -1,0 +1,276 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle
+on the same seeded inputs.  Codes must be the exact argmin outside the 1e-5
+relative near-tie window; reconstructions and EMA codebooks must agree to 1e-3
+(plus, for 16-bit outputs, half an ulp of the output type)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2410_15704_b200 as rvq
+import rvq_synth
+from helpers import (DT, RECON_TOL, assert_codes_match, assert_recon_match, assert_std_match,
+                     codes_to_device, codes_to_numpy, config_of, gpu_decode, gpu_encode, x_to_device)
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_rows(n, k, seed):
+    return np.sort(np.random.default_rng(seed).choice(n, size=min(k, n), replace=False))
+
+
+# ---------------------------------------------------------------- the five workloads
+
+def test_tiny_encode_decode():
+    w = rvq_synth.tiny()
+    cfg = config_of(w)
+    codes, std_bits, st, b = gpu_encode(cfg, x_to_device(w.x, cfg.x_dtype), w.n, w.codebooks)
+    ties = assert_codes_match(w.x, codes, w.codebooks, w.layout)
+    assert_std_match(w.x, std_bits)
+    ref = oracle.encode(w.x, w.codebooks, w.group_dim, w.layout)
+    assert np.mean(ref["codes"] != codes) < 1e-3            # free-running agreement
+    assert st["degenerate_vectors"] == 0 and st["wait_timeouts"] == 0
+    got, _ = gpu_decode(cfg, ref["codes"], ref["std_bits"], w.codebooks, w.n)
+    err = assert_recon_match(got, ref["codes"], ref["std_bits"], w.codebooks, w.dim, w.layout, cfg.x_dtype)
+    print(f"tiny: near ties {ties}, decode max-abs {err:.2e}")
+
+
+def test_key_cache_encode_full_size():
+    w = rvq_synth.key_cache()
+    cfg = config_of(w)
+    codes, std_bits, st, _ = gpu_encode(cfg, x_to_device(w.x, cfg.x_dtype), w.n, w.codebooks)
+    ties = assert_codes_match(w.x, codes, w.codebooks, w.layout)
+    changed = assert_std_match(w.x, std_bits)
+    assert st["wait_timeouts"] == 0
+    print(f"key_cache: near ties {ties} of {codes.size}, std off by one ulp {changed:.2e}, status {st}")
+
+
+def test_value_cache_encode_decode_packed():
+    w = rvq_synth.value_cache()
+    cfg = config_of(w)
+    assert cfg.code_bits == 11 and rvq.rvq_code_bytes(cfg) == 44
+    codes, std_bits, st, b = gpu_encode(cfg, x_to_device(w.x, cfg.x_dtype), w.n, w.codebooks)
+    rows = sample_rows(w.n, 6000, 3)
+    ties = assert_codes_match(w.x, codes, w.codebooks, w.layout, sample=rows)
+    assert_std_match(w.x, std_bits)
+    assert codes.min() >= 0 and codes.max() < w.codebook_size
+    got, _ = gpu_decode(cfg, codes, std_bits, w.codebooks, w.n)
+    err = assert_recon_match(got, codes, std_bits, w.codebooks, w.dim, w.layout, cfg.x_dtype)
+    # reconstruction error is what the quantizer leaves, far below the signal
+    rel = np.mean((got - w.x) ** 2) / np.mean(w.x.astype(np.float64) ** 2)
+    assert rel < 0.2
+    print(f"value_cache: sampled near ties {ties}, decode max-abs {err:.2e}, relative MSE {rel:.3f}")
+
+
+@pytest.mark.parametrize("layout", [rvq_synth.CONTIGUOUS, rvq_synth.STRIDED])
+def test_decode_bandwidth_full_size(layout):
+    w = rvq_synth.decode_bandwidth(layout=layout)
+    cfg = config_of(w)
+    got, st = gpu_decode(cfg, w.codes, w.std_bits, w.codebooks, w.n)
+    rows = sample_rows(w.n, 100000, 4)
+    err = assert_recon_match(got, w.codes, w.std_bits, w.codebooks, w.dim, layout, cfg.x_dtype, rows=rows)
+    cfg32 = config_of(w, x_dtype=rvq.F32)
+    sub = np.arange(0, 70001)
+    got32, _ = gpu_decode(cfg32, w.codes[sub], w.std_bits[sub], w.codebooks, len(sub))
+    err32 = assert_recon_match(got32, w.codes[sub], w.std_bits[sub], w.codebooks, w.dim, layout, rvq.F32)
+    assert st["bad_codes"] == 0
+    print(f"decode layout {layout}: bf16 max-abs {err:.2e}, fp32 max-abs {err32:.2e}")
+
+
+def test_decode_head_major_tiles():
+    """Output rows written through a row stride: [head][token][dim] tiles."""
+    w = rvq_synth.decode_bandwidth(tokens=1024)
+    cfg = config_of(w)
+    got, _ = gpu_decode(cfg, w.codes, w.std_bits, w.codebooks, w.n, row_stride=160)
+    assert np.all(got[:, 128:] == 7.0)                       # padding untouched
+    assert_recon_match(got, w.codes, w.std_bits, w.codebooks, w.dim, w.layout, cfg.x_dtype)
+
+
+def run_ema_steps(w, steps, tokens_check=True):
+    cfg = config_of(w)
+    x_dev = x_to_device(w.x, cfg.x_dtype)
+    b = rvq.alloc_buffers(cfg, w.n, w.codebooks)
+    R, K, gd = w.codebooks.shape
+    ema_count = torch.ones(R, K, device="cuda")
+    ema_sum = b.codebooks.clone()
+    batch = torch.empty(R, K, device="cuda")
+    worst = 0.0
+    for step in range(steps):
+        cb_before = b.codebooks.cpu().numpy()
+        n_before = ema_count.cpu().numpy().astype(np.float64)
+        m_before = ema_sum.cpu().numpy().astype(np.float64)
+        rvq.rvq_prepare_codebooks(cfg, b.codebooks, b.prepared)
+        rvq.rvq_encode(cfg, x_dev, w.n, w.dim, b.codebooks, b.prepared, b.codes, b.std, b.workspace,
+                       b.workspace_bytes, b.status)
+        rvq.rvq_ema_update(cfg, x_dev, w.n, w.dim, b.codes, b.codebooks, ema_count, ema_sum, batch,
+                           w.decay, w.eps, b.workspace, b.workspace_bytes, b.status)
+        torch.cuda.synchronize()
+        codes = codes_to_numpy(cfg, b.codes, w.n)
+        rows = None if w.n <= 20000 else sample_rows(w.n, 4000, 10 + step)
+        assert_codes_match(w.x, codes, cb_before, w.layout, sample=rows)
+        # teacher-forced: the oracle's update from the same codes and the same state
+        ref = oracle.ema_update(w.x, codes, cb_before, n_before, m_before, w.decay, w.eps, w.layout)
+        assert np.array_equal(batch.cpu().numpy().astype(np.int64), ref["count"].astype(np.int64))
+        assert int(batch.sum().item()) == w.n * w.groups * R
+        e_cb = np.abs(b.codebooks.cpu().numpy() - ref["codebooks"]).max()
+        e_n = np.abs(ema_count.cpu().numpy() - ref["ema_count"]).max()
+        e_m = np.abs(ema_sum.cpu().numpy() - ref["ema_sum"]).max()
+        assert e_cb <= RECON_TOL and e_m <= RECON_TOL and e_n <= 1e-3 * max(1.0, ref["ema_count"].max())
+        worst = max(worst, e_cb)
+    st = rvq.read_status(b.status)
+    assert st["bad_codes"] == 0 and st["wait_timeouts"] == 0
+    return worst
+
+
+def test_ema_learning_three_steps_reduced():
+    w = rvq_synth.ema_learning(tokens=2048, steps=3)
+    worst = run_ema_steps(w, 3)
+    print(f"ema (16384 vectors, 3 steps): codebook max-abs {worst:.2e}")
+
+
+def test_ema_learning_full_size_one_step():
+    w = rvq_synth.ema_learning()
+    worst = run_ema_steps(w, 1)
+    print(f"ema (1048576 vectors, 1 step): codebook max-abs {worst:.2e}")
+
+
+def test_ema_resume_equals_straight_run():
+    """5 steps + save + load + 5 steps equals 10 straight steps (same codes, state within tolerance)."""
+    w = rvq_synth.ema_learning(tokens=256)
+    cfg = config_of(w)
+    x_dev = x_to_device(w.x, cfg.x_dtype)
+
+    def run(steps, state=None):
+        b = rvq.alloc_buffers(cfg, w.n, w.codebooks if state is None else state[0])
+        n_ = torch.ones_like(b.codebooks[..., 0]) if state is None else state[1].clone().cuda()
+        m_ = b.codebooks.clone() if state is None else state[2].clone().cuda()
+        for _ in range(steps):
+            rvq.rvq_prepare_codebooks(cfg, b.codebooks, b.prepared)
+            rvq.rvq_encode(cfg, x_dev, w.n, w.dim, b.codebooks, b.prepared, b.codes, b.std, b.workspace,
+                           b.workspace_bytes, b.status)
+            rvq.rvq_ema_update(cfg, x_dev, w.n, w.dim, b.codes, b.codebooks, n_, m_, None, w.decay, w.eps,
+                               b.workspace, b.workspace_bytes, b.status)
+        torch.cuda.synchronize()
+        return b.codebooks.cpu(), n_.cpu(), m_.cpu()
+
+    straight = run(10)
+    resumed = run(5, run(5))
+    for a, c in zip(straight, resumed):
+        assert torch.max(torch.abs(a - c)).item() <= 1e-4
+
+
+# ---------------------------------------------------------------- shapes and edge cases
+
+@pytest.mark.parametrize("n", [0, 1, 31, 33, 257])
+def test_ragged_sizes(n):
+    w = rvq_synth.tiny(300)
+    cfg = config_of(w, x_dtype=rvq.F32)
+    x = w.x[:n]
+    xd = x_to_device(w.x, cfg.x_dtype)[:max(n, 1)]
+    codes, std_bits, st, b = gpu_encode(cfg, xd, n, w.codebooks)
+    if n:
+        assert_codes_match(x, codes, w.codebooks, w.layout)
+        assert_std_match(x, std_bits)
+    got, _ = gpu_decode(cfg, codes, std_bits, w.codebooks, n)
+    if n:
+        assert_recon_match(got, codes, std_bits, w.codebooks, w.dim, w.layout, cfg.x_dtype)
+
+
+@pytest.mark.parametrize("dim,gd,R,K,layout,dtype,bits,ddof", [
+    (128, 32, 4, 1024, 1, "bf16", 10, 0),
+    (128, 32, 6, 2048, 0, "f16", 11, 0),
+    (128, 32, 8, 300, 1, "f32", 9, 1),
+    (128, 32, 1, 256, 0, "bf16", 16, 0),
+    (256, 32, 8, 512, 1, "bf16", 16, 0),
+    (128, 16, 8, 256, 1, "bf16", 8, 0),
+    (128, 64, 3, 128, 0, "f32", 16, 0),
+    (64, 8, 16, 64, 1, "f16", 6, 1),
+])
+def test_shape_grid(dim, gd, R, K, layout, dtype, bits, ddof):
+    g = np.random.default_rng(dim + gd + R + K)
+    n = 777
+    x = g.normal(size=(n, dim)) * g.uniform(0.3, 4.0, size=(1, dim))
+    xt = torch.from_numpy(x).to(rvq.TORCH_DTYPE[DT[dtype]])
+    x = xt.float().numpy()                                         # exactly representable values
+    cb = np.stack([g.normal(scale=0.8 ** r, size=(K, gd)) for r in range(R)]).astype(np.float32)
+    cfg = rvq.make_config(dim, gd, layout, R, K, bits, DT[dtype], ddof)
+    codes, std_bits, st, _ = gpu_encode(cfg, xt.cuda(), n, cb)
+    assert_codes_match(x, codes, cb, layout, ddof)
+    assert_std_match(x, std_bits, ddof)
+    got, _ = gpu_decode(cfg, codes, std_bits, cb, n)
+    assert_recon_match(got, codes, std_bits, cb, dim, layout, cfg.x_dtype)
+    # one EMA step from these codes
+    b = rvq.alloc_buffers(cfg, n, cb)
+    cnt, msum = torch.ones(R, K, device="cuda"), b.codebooks.clone()
+    rvq.rvq_ema_update(cfg, xt.cuda(), n, dim, codes_to_device(cfg, codes), b.codebooks, cnt, msum, None,
+                       0.9, 1e-5, b.workspace, b.workspace_bytes, b.status)
+    torch.cuda.synchronize()
+    ref = oracle.ema_update(x, codes, cb, np.ones((R, K)), cb.astype(np.float64), 0.9, 1e-5, layout, ddof)
+    assert np.abs(b.codebooks.cpu().numpy() - ref["codebooks"]).max() <= RECON_TOL
+
+
+def test_row_stride_on_input():
+    w = rvq_synth.key_cache(tokens=64)
+    cfg = config_of(w)
+    xd = x_to_device(w.x, cfg.x_dtype, row_stride=136)
+    codes, std_bits, _, _ = gpu_encode(cfg, xd, w.n, w.codebooks, row_stride=136)
+    assert_codes_match(w.x, codes, w.codebooks, w.layout)
+
+
+def test_degenerate_vectors_and_bad_codes():
+    w = rvq_synth.tiny(64)
+    cfg = config_of(w)
+    x = w.x.copy()
+    x[3] = 0.0
+    x[9] = -2.5
+    x[17, 4] = np.nan
+    x[40, 100] = np.inf
+    codes, std_bits, st, b = gpu_encode(cfg, x_to_device(x, cfg.x_dtype), w.n, w.codebooks)
+    assert st["degenerate_vectors"] == 4
+    for v in (3, 9, 17, 40):
+        assert std_bits[v] == 0 and not codes[v].any()
+    keep = np.setdiff1d(np.arange(64), [3, 9, 17, 40])
+    assert_codes_match(x[keep], codes[keep], w.codebooks, w.layout)
+    got, _ = gpu_decode(cfg, codes, std_bits, w.codebooks, w.n)
+    assert np.all(got[[3, 9, 17, 40]] == 0.0)
+    bad = codes.copy()
+    bad[5, 1, 2] = 60000
+    got, st2 = gpu_decode(cfg, bad, std_bits, w.codebooks, w.n)
+    assert st2["bad_codes"] >= 1 and np.all(np.isfinite(got))
+    fixed = bad.copy()
+    fixed[5, 1, 2] = 0
+    assert_recon_match(got, fixed, std_bits, w.codebooks, w.dim, w.layout, cfg.x_dtype)
+
+
+def test_scale_invariance_on_gpu():
+    w = rvq_synth.tiny(256)
+    cfg = config_of(w)
+    a, sa, _, _ = gpu_encode(cfg, x_to_device(w.x, cfg.x_dtype), w.n, w.codebooks)
+    c, sc, _, _ = gpu_encode(cfg, x_to_device(w.x * 8.0, cfg.x_dtype), w.n, w.codebooks)
+    assert np.array_equal(a, c)
+    np.testing.assert_array_equal(oracle.f16_value(sc), 8.0 * oracle.f16_value(sa))
+
+
+def test_exact_reconstruction_codebooks():
+    """Inputs that are sums of codewords with wide gaps come back exactly."""
+    import itertools
+    R, K, gd, G, n = 8, 64, 32, 4, 500
+    pats = [p for p in itertools.product([1, -1], repeat=4) if sum(p) == 0]
+    cb = np.zeros((R, K, gd))
+    for r in range(R):
+        for j in range(K):
+            cb[r, j, 4 * r:4 * r + 4] = np.array(pats[j % 6]) * 4.0 ** -r * (1.0 if j < 6 else 3.0 + j)
+    var = sum(4 * 16.0 ** -r for r in range(R)) / gd
+    cb = (cb / np.sqrt(var)).astype(np.float32)
+    g = np.random.default_rng(0)
+    codes = g.integers(0, 6, size=(n, G, R))
+    z = np.zeros((n, G * gd), dtype=np.float64)
+    for g_ in range(G):
+        for r in range(R):
+            z[:, g_ * gd:(g_ + 1) * gd] += cb[r, codes[:, g_, r]].astype(np.float64)
+    x = (2.0 * z).astype(np.float32)
+    cfg = rvq.make_config(G * gd, gd, 0, R, K, 16, rvq.F32, 0)
+    got_codes, std_bits, _, _ = gpu_encode(cfg, torch.from_numpy(x).cuda(), n, cb)
+    assert np.array_equal(got_codes, codes)
+    got, _ = gpu_decode(cfg, got_codes, std_bits, cb, n)
+    assert np.abs(got - x).max() <= 2e-3          # std ~2 rounds to half precision: 2 * 2^-11 relative

@@ -134,6 +134,17 @@ int rvq_encode(const rvq_config *cfg /* host */, const void *x, int64_t n, int64
                void *stream /* cudaStream_t */);
 
 /*
+ * The same encode computed entirely in float32 on the CUDA cores (every
+ * distance in the direct form sum((z - e)^2), no tensor cores, no prepared
+ * operands).  Same arguments and results as rvq_encode; an order of magnitude
+ * slower.  It serves shapes the tensor-core kernel does not cover and is the
+ * on-device cross-check of rvq_encode: both emit identical codes.
+ */
+int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
+                     const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+                     rvq_status *status, void *stream /* cudaStream_t */);
+
+/*
  * Decode (Section 2.2, last sentence; Section 3.2).  For every head vector and
  * channel c = channel(g, i): x_out[c] = std * sum_r C_r[code[g][r]][i], summed
  * in float32 in stage order and rounded once to x_dtype.

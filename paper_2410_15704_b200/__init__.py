@@ -56,6 +56,8 @@ def _load() -> ctypes.CDLL:
     lib.rvq_prepare_codebooks.argtypes = [cfgp, vp, vp, vp]
     lib.rvq_encode.restype = ctypes.c_int
     lib.rvq_encode.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.rvq_encode_exact.restype = ctypes.c_int
+    lib.rvq_encode_exact.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp]
     lib.rvq_decode.restype = ctypes.c_int
     lib.rvq_decode.argtypes = [cfgp, vp, vp, i64, vp, vp, vp, i64, vp, vp]
     lib.rvq_ema_update.restype = ctypes.c_int
@@ -71,7 +73,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 
-EXPORTS = ("rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
+EXPORTS = ("rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
            "rvq_prepare_codebooks", "rvq_workspace_bytes", "rvq_encode", "rvq_decode",
            "rvq_ema_update")
 
@@ -134,6 +136,15 @@ def rvq_encode(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, wor
                         _stream(stream))
     if check:
         _check(rc, "rvq_encode")
+    return rc
+
+
+def rvq_encode_exact(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status=None,
+                     stream=None, check=True) -> int:
+    rc = lib.rvq_encode_exact(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
+                              _ptr(codes), _ptr(std_f16), _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_encode_exact")
     return rc
 
 

@@ -99,9 +99,9 @@ size_t rvq_workspace_bytes(const rvq_config *cfg, int64_t n)
     return make_shape(cfg, &s) == RVQ_OK ? ema_workspace_bytes(s) : 0;
 }
 
-int rvq_encode(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
-               const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-               void *workspace, size_t workspace_bytes, rvq_status *status, void *stream)
+static int encode_common(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                         const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+                         rvq_status *status, void *stream, bool allow_tensor)
 {
     Shape s;
     int rc = make_shape(cfg, &s);
@@ -109,8 +109,25 @@ int rvq_encode(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_st
     if ((rc = check_rows(s, x, n, x_row_stride)) != RVQ_OK) return rc;
     if (!codebooks || !prepared || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
     if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
-    (void)workspace; (void)workspace_bytes;
+    if (allow_tensor && encode_tensor_supported(s))
+        return launch_encode_tensor(s, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status,
+                                    (cudaStream_t)stream);
     return launch_encode_scalar(s, x, n, x_row_stride, codebooks, codes, std_f16, status, (cudaStream_t)stream);
+}
+
+int rvq_encode(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+               const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+               void *workspace, size_t workspace_bytes, rvq_status *status, void *stream)
+{
+    (void)workspace; (void)workspace_bytes;
+    return encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, stream, true);
+}
+
+int rvq_encode_exact(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                     const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+                     rvq_status *status, void *stream)
+{
+    return encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, stream, false);
 }
 
 int rvq_decode(const rvq_config *cfg, const void *codes, const uint16_t *std_f16, int64_t n,

@@ -1,0 +1,487 @@
+// Tensor-core encode for group_dim 32 (Section 2.2, Algorithm 1).
+//
+// One persistent CTA per SM works on passes of 512 group rows (four tiles of 128
+// rows, one row per thread, 16 epilogue warps) plus one control warp.
+//   - Scores ||e||^2 - 2 z.e of a 128-row tile against 128 codewords are one
+//     tcgen05.mma chain (M=128, N=128, three K=16 steps over the 48-deep
+//     operands described in prepare.cu), accumulated in float32 in TMEM.
+//   - The B operand (256 codewords per slot) streams from the prepared block
+//     through a ring of shared-memory slots filled by cp.async.bulk; every
+//     slot serves all four tiles.
+//   - Epilogue threads read their row's 128 scores with tcgen05.ld and keep
+//     (i) the minimum of every 32-column block that comes within the error
+//     window of the running minimum, and (ii) the minimum per 3-column cell
+//     position over all blocks.  Any column that could be the exact argmin lies
+//     in a listed block at a listed cell position; those few columns are
+//     re-scored exactly in float32 against the float32 codebook (direct form,
+//     lowest index on ties), so the emitted code is the exact-L2 choice.
+//   - The residual stays in registers across all R stages; x is read once and
+//     only codes and the half-precision deviation are written.
+// Every wait is bounded; a wait that gives up sets status->wait_timeouts and
+// the kernel drains and returns.
+#include "prepared.cuh"
+
+namespace rvq {
+
+namespace {
+
+constexpr int kTiles = 4;
+constexpr int kRowsPerPass = 128 * kTiles;
+constexpr int kEpiThreads = kRowsPerPass;
+constexpr int kThreads = kEpiThreads + 32;
+constexpr int kRing = 4;                                  // operand slots in flight
+constexpr int kATileBytes = kSlotCells * 128 * 16;        // 12288
+constexpr int kListCap = 8;
+constexpr uint32_t kWaitLimit = 4u * 1000u * 1000u;
+
+constexpr int kOffB = 0;
+constexpr int kOffA = kOffB + kRing * kSlotBytes;                    //  98304
+constexpr int kOffListV = kOffA + kTiles * kATileBytes;              // 147456
+constexpr int kOffListI = kOffListV + kListCap * kRowsPerPass * 4;   // 163840
+constexpr int kOffCodes = kOffListI + kListCap * kRowsPerPass * 2;   // 172032
+constexpr int kOffBars = kOffCodes + kRowsPerPass * 16 * 2;          // 188416
+constexpr int kSmemBytes = kOffBars + 256;
+
+// barrier slots
+constexpr int kBarFull = 0, kBarEmpty = kRing, kBarAReady = 2 * kRing, kBarAccFull = 2 * kRing + kTiles,
+              kBarAccFree = 2 * kRing + 2 * kTiles, kNumBars = 2 * kRing + 3 * kTiles;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait; returns false (and raises the CTA's abort flag) when it gives up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    return false;
+}
+
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    // K-major, no swizzle: 8x16-byte core matrices; LBO steps along the
+    // contraction, SBO along rows; descriptor version 1.
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | ((uint64_t)1 << 46);
+}
+
+__device__ __forceinline__ void mma_f16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ float min3(float a, float b, float c)
+{
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t u[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+                   "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+                   "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+                   "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(u[i]);
+}
+
+// Exact squared distance, direct form, same operation order as the scalar kernel.
+__device__ __forceinline__ float exact_distance(const float (&z)[32], const float *__restrict__ e)
+{
+    float acc = 0.0f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const float4 ev = __ldg(reinterpret_cast<const float4 *>(e) + q);
+        const float t0 = z[4 * q] - ev.x, t1 = z[4 * q + 1] - ev.y, t2 = z[4 * q + 2] - ev.z, t3 = z[4 * q + 3] - ev.w;
+        acc = fmaf(t0, t0, acc); acc = fmaf(t1, t1, acc); acc = fmaf(t2, t2, acc); acc = fmaf(t3, t3, acc);
+    }
+    return acc;
+}
+
+struct Params {
+    Shape s;
+    const void *x;
+    int64_t n, stride;
+    const float *cb;
+    const uint8_t *prepared;
+    void *codes;
+    uint16_t *std16;
+    rvq_status *st;
+    int passes;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+encode_tensor_kernel(const Params p)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kOffBars);
+    uint32_t *tmem_word = reinterpret_cast<uint32_t *>(smem + kOffBars + kNumBars * 8);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kOffBars + kNumBars * 8 + 4);
+
+    const Shape &s = p.s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int S = slots_per_stage(s.K);
+    const int my_passes = (p.passes - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const StageParams *sp = reinterpret_cast<const StageParams *>(p.prepared + kPreparedParamsOffset);
+    const uint8_t *image = p.prepared + kPreparedImageOffset;
+    const uint32_t bar0 = smem_u32(bars);
+    auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    if (tid == 0) {
+        for (int i = 0; i < kRing; ++i) { mbar_init(BAR(kBarFull + i), 1); mbar_init(BAR(kBarEmpty + i), 1); }
+        for (int t = 0; t < kTiles; ++t) {
+            mbar_init(BAR(kBarAReady + t), 128); mbar_init(BAR(kBarAccFull + t), 1); mbar_init(BAR(kBarAccFree + t), 128);
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kEpiThreads / 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_word)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    // constant part of every A row: cell 4 = (1, 1, 1, 0...), cell 5 = 0
+    if (tid < kEpiThreads) {
+        const int tile = tid >> 7, row = tid & 127;
+        uint8_t *a = smem + kOffA + tile * kATileBytes + row * 16;
+        *reinterpret_cast<uint4 *>(a + 4 * 2048) = make_uint4(0x3C003C00u, 0x00003C00u, 0u, 0u);
+        *reinterpret_cast<uint4 *>(a + 5 * 2048) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_word;
+
+    if (warp == kEpiThreads / 32) {
+        // ------------------------------------------------------------ control warp
+        if (lane == 0 && my_passes > 0) {
+            const uint32_t total = (uint32_t)my_passes * (uint32_t)s.R * (uint32_t)S;
+            const uint32_t idesc = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);   // f16 x f16 -> f32, M=N=128
+            uint32_t n_load = 0;
+            bool ok = true;
+            for (uint32_t q = 0; q < total && ok; ++q) {
+                while (ok && n_load < total && n_load < q + kRing - 1) {
+                    const uint32_t slot = n_load % kRing, use = n_load / kRing;
+                    if (use > 0) ok = mbar_wait(BAR(kBarEmpty + slot), (use - 1) & 1u, abort_flag);
+                    if (!ok) break;
+                    const uint32_t rs = n_load % ((uint32_t)s.R * S);      // (stage, slot-in-stage), row-major
+                    mbar_expect_tx(BAR(kBarFull + slot), kSlotBytes);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(smem + kOffB + slot * kSlotBytes)), "l"(image + (size_t)rs * kSlotBytes),
+                                   "r"((uint32_t)kSlotBytes), "r"(BAR(kBarFull + slot)) : "memory");
+                    ++n_load;
+                }
+                if (!ok) break;
+                const uint32_t slot = q % kRing, use = q / kRing;
+                ok = mbar_wait(BAR(kBarFull + slot), use & 1u, abort_flag);
+                const uint32_t stage_global = q / S, s_in = q % S;
+                const uint32_t b_base = smem_u32(smem + kOffB + slot * kSlotBytes);
+                for (int h = 0; h < 2 && ok; ++h) {
+                    for (int t = 0; t < kTiles && ok; ++t) {
+                        if (s_in == 0 && h == 0) ok = mbar_wait(BAR(kBarAReady + t), stage_global & 1u, abort_flag);
+                        const uint32_t c = 2 * q + h;
+                        if (ok && c > 0) ok = mbar_wait(BAR(kBarAccFree + t), (c - 1) & 1u, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t a_base = smem_u32(smem + kOffA + t * kATileBytes);
+#pragma unroll
+                        for (int kk = 0; kk < 3; ++kk) {
+                            const uint64_t adesc = make_smem_desc(a_base + kk * 2 * 2048, 2048, 128);
+                            const uint64_t bdesc = make_smem_desc(b_base + h * 128 * 16 + kk * 2 * (kSlotCodewords * 16),
+                                                                  kSlotCodewords * 16, 128);
+                            mma_f16_ss(tmem + t * 128, adesc, bdesc, idesc, kk > 0);
+                        }
+                        mma_commit(BAR(kBarAccFull + t));
+                    }
+                }
+                if (ok) mma_commit(BAR(kBarEmpty + slot));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int tile = warp >> 2, q4 = warp & 3;
+        const int rloc = tile * 128 + q4 * 32 + lane;
+        const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)tile * 128u;
+        uint8_t *a_row = smem + kOffA + tile * kATileBytes + (q4 * 32 + lane) * 16;
+        float *list_v = reinterpret_cast<float *>(smem + kOffListV) + rloc;              // [e][row]
+        uint16_t *list_i = reinterpret_cast<uint16_t *>(smem + kOffListI) + rloc;         // [e][row]
+        uint16_t *codes_s = reinterpret_cast<uint16_t *>(smem + kOffCodes);                // [row][R]
+        const int G = s.G;
+        uint32_t chunk_use = 0, stage_global = 0;
+        uint32_t n_rescored = 0, n_exhaustive = 0, n_degenerate = 0, n_stdrange = 0;
+        bool ok = true;
+
+        for (int pass = 0; pass < my_passes && ok; ++pass) {
+            const int64_t row0 = ((int64_t)blockIdx.x + (int64_t)pass * gridDim.x) * kRowsPerPass;
+            const int64_t grow = row0 + rloc;
+            const int64_t v = grow / G;
+            const int g = (int)(grow - v * G);
+            const bool valid = v < p.n;
+
+            float z[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                z[i] = valid ? load_as_float(p.x, v * p.stride + channel_of(s.layout, G, 32, g, i), s.dtype) : 0.0f;
+            // deviation over the G lanes of this head vector, same summation order as the scalar kernel
+            float dev;
+            {
+                float a = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) a += z[i];
+                const int base = lane - g;
+                float mu = 0.0f;
+                for (int k = 0; k < G; ++k) mu += __shfl_sync(0xFFFFFFFFu, a, base + k);
+                mu /= (float)s.dim;
+                float b = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) b += (z[i] - mu) * (z[i] - mu);
+                float ss = 0.0f;
+                for (int k = 0; k < G; ++k) ss += __shfl_sync(0xFFFFFFFFu, b, base + k);
+                dev = sqrtf(ss / (float)(s.dim - s.ddof));
+            }
+            const bool deg = deviation_is_degenerate(dev) || !valid;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) z[i] = deg ? 0.0f : z[i] / dev;
+            if (valid && g == 0) {
+                const uint16_t hb = deviation_is_degenerate(dev) ? (uint16_t)0 : __half_as_ushort(__float2half_rn(dev));
+                p.std16[v] = hb;
+                if (deviation_is_degenerate(dev)) ++n_degenerate;
+                else if ((hb & 0x7FFFu) == 0 || (hb & 0x7FFFu) >= 0x7C00u) ++n_stdrange;
+            }
+
+#pragma unroll 1
+            for (int r = 0; r < s.R && ok; ++r) {
+                const StageParams prm = sp[r];
+                const float *cbr = p.cb + (size_t)r * s.K * 32;
+                // scaled half-precision copy of the residual -> A operand row; error window of this row
+                float zz = 0.0f, zmax = 0.0f;
+                {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float z0 = z[2 * i] * prm.scale, z1 = z[2 * i + 1] * prm.scale;
+                        zz = fmaf(z0, z0, zz); zz = fmaf(z1, z1, zz);
+                        zmax = fmaxf(zmax, fmaxf(fabsf(z0), fabsf(z1)));
+                        const __half2 h2 = __floats2half2_rn(z0, z1);
+                        pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        *reinterpret_cast<uint4 *>(a_row + c * 2048) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(BAR(kBarAReady + tile));
+                ++stage_global;
+                const float win = 2.125f * (prm.a * sqrtf(zz) * 1.0001f + prm.b);    // 2 * bound, with slack for this arithmetic
+                const bool force_scan = !(zmax < 60000.0f) || !(win < INFINITY);
+
+                float m1 = INFINITY, thr = INFINITY;
+                int cnt = 0;
+                float d[11];
+#pragma unroll
+                for (int q = 0; q < 11; ++q) d[q] = INFINITY;
+
+                const int chunks = 2 * S;
+#pragma unroll 1
+                for (int c = 0; c < chunks && ok; ++c) {
+                    ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag);
+                    ok = __all_sync(0xFFFFFFFFu, ok);          // tcgen05.ld below needs the whole warp
+                    ++chunk_use;
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int blk = 0; blk < 4; ++blk) {
+                        float sc[32];
+                        tmem_ld32(taddr + blk * 32, sc);
+                        if (blk == 3) {
+                            tc_fence_before();
+                            mbar_arrive(BAR(kBarAccFree + tile));
+                        }
+                        float t[11];
+#pragma unroll
+                        for (int q = 0; q < 10; ++q) t[q] = min3(sc[3 * q], sc[3 * q + 1], sc[3 * q + 2]);
+                        t[10] = fminf(sc[30], sc[31]);
+                        float cb_min = fminf(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])),
+                                             fminf(t[9], t[10]));
+#pragma unroll
+                        for (int q = 0; q < 11; ++q) d[q] = fminf(d[q], t[q]);
+                        if (cb_min <= thr) {
+                            m1 = fminf(m1, cb_min);
+                            thr = m1 + win;
+                            if (cnt == kListCap) {
+                                // drop entries that fell out of the window as the minimum came down
+                                int keep = 0;
+                                for (int e = 0; e < kListCap; ++e) {
+                                    const float fv = list_v[e * kRowsPerPass];
+                                    const uint16_t fi = list_i[e * kRowsPerPass];
+                                    if (fv <= thr) { list_v[keep * kRowsPerPass] = fv; list_i[keep * kRowsPerPass] = fi; ++keep; }
+                                }
+                                cnt = keep;
+                            }
+                            if (cnt < kListCap) {
+                                list_v[cnt * kRowsPerPass] = cb_min;
+                                list_i[cnt * kRowsPerPass] = (uint16_t)(c * 4 + blk);
+                                ++cnt;
+                            } else {
+                                cnt = kListCap + 1;      // more candidates than the list holds: scan everything
+                            }
+                        }
+                    }
+                }
+                if (!ok) break;
+
+                // ---- stage end: exact choice among the columns that can still be the argmin
+                int bj = 0;
+                if (!deg) {
+                    float best = INFINITY;
+                    const float lim = m1 + win;
+                    if (force_scan || cnt == 0 || cnt > kListCap) {
+                        ++n_exhaustive;
+                        for (int j = 0; j < s.K; ++j) {
+                            const float dj = exact_distance(z, cbr + (size_t)j * 32);
+                            if (dj < best) { best = dj; bj = j; }
+                        }
+                    } else {
+                        int listed = 0;
+                        for (int e = 0; e < cnt; ++e) {
+                            if (!(list_v[e * kRowsPerPass] <= lim)) continue;
+                            ++listed;
+                            const int col0 = (int)list_i[e * kRowsPerPass] * 32;
+#pragma unroll
+                            for (int q = 0; q < 11; ++q) {
+                                if (!(d[q] <= lim)) continue;
+                                for (int k = 0; k < 3; ++k) {
+                                    const int j = col0 + 3 * q + k;
+                                    if (3 * q + k >= 32 || j >= s.K) continue;
+                                    const float dj = exact_distance(z, cbr + (size_t)j * 32);
+                                    if (dj < best) { best = dj; bj = j; }      // columns visited in ascending order
+                                }
+                            }
+                        }
+                        int cells = 0;
+#pragma unroll
+                        for (int q = 0; q < 11; ++q) cells += (d[q] <= lim) ? 1 : 0;
+                        if (listed * cells > 1) ++n_rescored;
+                    }
+                    const float4 *e4 = reinterpret_cast<const float4 *>(cbr + (size_t)bj * 32);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 ev = __ldg(e4 + q);
+                        z[4 * q] -= ev.x; z[4 * q + 1] -= ev.y; z[4 * q + 2] -= ev.z; z[4 * q + 3] -= ev.w;
+                    }
+                }
+                codes_s[rloc * 16 + r] = (uint16_t)bj;
+            }
+            if (!ok) break;
+
+            // ---- emit the codes of this pass (Section 3.2 storage)
+            __syncwarp();
+            if (s.bits == 16) {
+                if (valid) {
+                    uint16_t *o = reinterpret_cast<uint16_t *>(p.codes) + (v * G + g) * s.R;
+                    if (s.R == 8) {
+                        *reinterpret_cast<uint4 *>(o) = *reinterpret_cast<const uint4 *>(codes_s + rloc * 16);
+                    } else {
+                        for (int r = 0; r < s.R; ++r) o[r] = codes_s[rloc * 16 + r];
+                    }
+                }
+            } else {
+                // lanes of this warp hold 32 / G whole head vectors; one 32-bit word per lane and step
+                const int words = s.code_bytes / 4, vec_per_warp = 32 / G;
+                const int wrow0 = rloc - lane;
+                for (int t = lane; t < vec_per_warp * words; t += 32) {
+                    const int vl = t / words, w = t - vl * words;
+                    const int64_t vv = (row0 + wrow0) / G + vl;
+                    if (vv >= p.n) continue;
+                    uint32_t word = 0;
+                    const int k_lo = (32 * w) / s.bits, k_hi = min(s.per_vector - 1, (32 * w + 31) / s.bits);
+                    for (int k = k_lo; k <= k_hi; ++k) {
+                        const int gg = k / s.R, rr = k - gg * s.R;
+                        const uint32_t val = codes_s[(wrow0 + vl * G + gg) * 16 + rr];
+                        const int sh = k * s.bits - 32 * w;
+                        word |= sh >= 0 ? (val << sh) : (val >> (-sh));
+                    }
+                    reinterpret_cast<uint32_t *>(p.codes)[vv * words + w] = word;
+                }
+            }
+            __syncwarp();
+        }
+        if (p.st) {
+            if (n_rescored) atomicAdd(&p.st->rescored_rows, n_rescored);
+            if (n_exhaustive) atomicAdd(&p.st->exhaustive_rows, n_exhaustive);
+            if (n_degenerate) atomicAdd(&p.st->degenerate_vectors, n_degenerate);
+            if (n_stdrange) atomicAdd(&p.st->std_out_of_half, n_stdrange);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kEpiThreads / 32) {
+        tc_fence_after();
+        if (lane == 0 && *abort_flag && p.st) atomicAdd(&p.st->wait_timeouts, 1u);
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
+    }
+}
+
+}  // namespace
+
+bool encode_tensor_supported(const Shape &s)
+{
+    return s.gd == 32 && s.G <= 32 && (s.G & (s.G - 1)) == 0 && slots_per_stage(s.K) * 8 <= 65535;
+}
+
+int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
+                         const void *prepared, void *codes, uint16_t *std16, rvq_status *st,
+                         cudaStream_t stream)
+{
+    if (n == 0) return RVQ_OK;
+    const int64_t rows = n * s.G;
+    const int64_t passes = (rows + kRowsPerPass - 1) / kRowsPerPass;
+    if (passes > 0x7FFFFFFF) return RVQ_ERR_UNSUPPORTED;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return RVQ_ERR_DEVICE;
+    if (cudaFuncSetAttribute(encode_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        return RVQ_ERR_LAUNCH;
+    Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)passes};
+    const int grid = (int)(passes < sms ? passes : sms);
+    encode_tensor_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);
+    return check_launch();
+}
+
+}  // namespace rvq

@@ -160,6 +160,39 @@ def test_ema_resume_equals_straight_run():
         assert torch.max(torch.abs(a - c)).item() <= 1e-4
 
 
+def test_tensor_encode_equals_exact_encode():
+    """The tensor-core encode and the all-float32 CUDA-core encode emit identical codes."""
+    for w in (rvq_synth.tiny(), rvq_synth.key_cache(tokens=1500), rvq_synth.value_cache(tokens=700)):
+        cfg = config_of(w)
+        xd = x_to_device(w.x, cfg.x_dtype)
+        codes, std_bits, st, b = gpu_encode(cfg, xd, w.n, w.codebooks)
+        b2 = rvq.alloc_buffers(cfg, w.n, w.codebooks)
+        rvq.rvq_encode_exact(cfg, xd, w.n, w.dim, b2.codebooks, b2.prepared, b2.codes, b2.std, b2.status)
+        torch.cuda.synchronize()
+        assert np.array_equal(codes, codes_to_numpy(cfg, b2.codes, w.n))
+        assert np.array_equal(std_bits, b2.std.cpu().numpy().view(np.uint16)[:w.n])
+        rows = w.n * w.groups * w.depth
+        print(f"{w.name}: re-scored {st['rescored_rows'] / rows:.4f} of row-stages, full scans {st['exhaustive_rows']}")
+        assert st["wait_timeouts"] == 0 and st["exhaustive_rows"] < 1e-3 * rows
+
+
+def test_tensor_encode_hostile_codebooks():
+    """Codebooks far outside the half-precision range, duplicates and zeros: still exact."""
+    g = np.random.default_rng(5)
+    n, R, K = 600, 3, 512
+    x = g.normal(size=(n, 128)).astype(np.float32)
+    cb = g.normal(size=(R, K, 32)).astype(np.float32)
+    cb[0, 100:110] = cb[0, 7]                 # duplicates: lowest index must win
+    cb[1] *= 1e-6                             # tiny stage
+    cb[2, :256] *= 3e4                        # huge spread inside one stage
+    cb[2, 300] = 0.0
+    cfg = rvq.make_config(128, 32, 0, R, K, 16, rvq.F32, 0)
+    codes, std_bits, st, _ = gpu_encode(cfg, torch.from_numpy(x).cuda(), n, cb)
+    assert_codes_match(x, codes, cb, 0)
+    assert not np.isin(codes[:, :, 0], np.arange(100, 110)).any()
+    print(f"hostile codebooks: status {st}")
+
+
 # ---------------------------------------------------------------- shapes and edge cases
 
 @pytest.mark.parametrize("n", [0, 1, 31, 33, 257])

@@ -3,9 +3,10 @@
 // One persistent CTA per SM works on passes of 512 group rows (four tiles of 128
 // rows, one row per thread, 16 epilogue warps) plus one control warp.
 //   - Scores ||e||^2 - 2 z.e of a 128-row tile against 128 codewords are one
-//     tcgen05.mma chain (M=128, N=128, three K=16 steps over the 48-deep
-//     operands described in prepare.cu), accumulated in float32 in TMEM.
-//   - The B operand (256 codewords per slot) streams from the prepared block
+//     tcgen05.mma chain (M=128, N=128, seven K=16 steps over the split
+//     half-precision operands described in prepare.cu), accumulated in float32
+//     in TMEM.
+//   - The B operand (128 codewords per slot) streams from the prepared block
 //     through a ring of shared-memory slots filled by cp.async.bulk; every
 //     slot serves all four tiles.
 //   - Epilogue threads read their row's 128 scores with tcgen05.ld and keep
@@ -30,15 +31,15 @@ constexpr int kRowsPerPass = 128 * kTiles;
 constexpr int kEpiThreads = kRowsPerPass;
 constexpr int kThreads = kEpiThreads + 32;
 constexpr int kRing = 4;                                  // operand slots in flight
-constexpr int kATileBytes = kSlotCells * 128 * 16;        // 12288
+constexpr int kATileBytes = kSlotCells * 128 * 16;        // 20480
 constexpr int kListCap = 8;
 constexpr uint32_t kWaitLimit = 4u * 1000u * 1000u;
 
 constexpr int kOffB = 0;
-constexpr int kOffA = kOffB + kRing * kSlotBytes;                    //  98304
-constexpr int kOffListV = kOffA + kTiles * kATileBytes;              // 147456
-constexpr int kOffListI = kOffListV + kListCap * kRowsPerPass * 4;   // 163840
-constexpr int kOffCodes = kOffListI + kListCap * kRowsPerPass * 2;   // 172032
+constexpr int kOffA = kOffB + kRing * kSlotBytes;                    //  81920
+constexpr int kOffListV = kOffA + kTiles * kATileBytes;              // 163840
+constexpr int kOffListI = kOffListV + (kListCap + 1) * kRowsPerPass * 4;   // 180224
+constexpr int kOffCodes = kOffListI + (kListCap + 1) * kRowsPerPass * 2;   // 172032
 constexpr int kOffBars = kOffCodes + kRowsPerPass * 16 * 2;          // 188416
 constexpr int kSmemBytes = kOffBars + 256;
 
@@ -145,6 +146,7 @@ struct Params {
     int passes;
 };
 
+// 17 warps are granted registers as 20 (whole groups of four): 96 per thread.
 __global__ void __launch_bounds__(kThreads, 1)
 encode_tensor_kernel(const Params p)
 {
@@ -174,12 +176,12 @@ encode_tensor_kernel(const Params p)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_word)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
-    // constant part of every A row: cell 4 = (1, 1, 1, 0...), cell 5 = 0
+    // constant part of every A row: cell 8 = (1, 1, 1, 0...), cell 9 = 0
     if (tid < kEpiThreads) {
         const int tile = tid >> 7, row = tid & 127;
         uint8_t *a = smem + kOffA + tile * kATileBytes + row * 16;
-        *reinterpret_cast<uint4 *>(a + 4 * 2048) = make_uint4(0x3C003C00u, 0x00003C00u, 0u, 0u);
-        *reinterpret_cast<uint4 *>(a + 5 * 2048) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4 *>(a + 8 * 2048) = make_uint4(0x3C003C00u, 0x00003C00u, 0u, 0u);
+        *reinterpret_cast<uint4 *>(a + 9 * 2048) = make_uint4(0u, 0u, 0u, 0u);
     }
     tc_fence_before();
     __syncthreads();
@@ -210,23 +212,23 @@ encode_tensor_kernel(const Params p)
                 ok = mbar_wait(BAR(kBarFull + slot), use & 1u, abort_flag);
                 const uint32_t stage_global = q / S, s_in = q % S;
                 const uint32_t b_base = smem_u32(smem + kOffB + slot * kSlotBytes);
-                for (int h = 0; h < 2 && ok; ++h) {
-                    for (int t = 0; t < kTiles && ok; ++t) {
-                        if (s_in == 0 && h == 0) ok = mbar_wait(BAR(kBarAReady + t), stage_global & 1u, abort_flag);
-                        const uint32_t c = 2 * q + h;
-                        if (ok && c > 0) ok = mbar_wait(BAR(kBarAccFree + t), (c - 1) & 1u, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t a_base = smem_u32(smem + kOffA + t * kATileBytes);
+                // (A cell pair, B cell pair) of the seven K=16 steps: hi.hi, hi.lo, lo.hi, 1.norm
+                constexpr int kStepA[7] = {0, 2, 0, 2, 4, 6, 8};
+                constexpr int kStepB[7] = {0, 2, 4, 6, 0, 2, 8};
+                for (int t = 0; t < kTiles && ok; ++t) {
+                    if (s_in == 0) ok = mbar_wait(BAR(kBarAReady + t), stage_global & 1u, abort_flag);
+                    if (ok && q > 0) ok = mbar_wait(BAR(kBarAccFree + t), (q - 1) & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_base = smem_u32(smem + kOffA + t * kATileBytes);
 #pragma unroll
-                        for (int kk = 0; kk < 3; ++kk) {
-                            const uint64_t adesc = make_smem_desc(a_base + kk * 2 * 2048, 2048, 128);
-                            const uint64_t bdesc = make_smem_desc(b_base + h * 128 * 16 + kk * 2 * (kSlotCodewords * 16),
-                                                                  kSlotCodewords * 16, 128);
-                            mma_f16_ss(tmem + t * 128, adesc, bdesc, idesc, kk > 0);
-                        }
-                        mma_commit(BAR(kBarAccFull + t));
+                    for (int kk = 0; kk < 7; ++kk) {
+                        const uint64_t adesc = make_smem_desc(a_base + kStepA[kk] * 2048, 2048, 128);
+                        const uint64_t bdesc = make_smem_desc(b_base + kStepB[kk] * (kSlotCodewords * 16),
+                                                              kSlotCodewords * 16, 128);
+                        mma_f16_ss(tmem + t * 128, adesc, bdesc, idesc, kk > 0);
                     }
+                    mma_commit(BAR(kBarAccFull + t));
                 }
                 if (ok) mma_commit(BAR(kBarEmpty + slot));
             }
@@ -290,18 +292,23 @@ encode_tensor_kernel(const Params p)
                 // scaled half-precision copy of the residual -> A operand row; error window of this row
                 float zz = 0.0f, zmax = 0.0f;
                 {
-                    uint32_t pk[16];
+                    uint32_t hi[16], lo[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const float z0 = z[2 * i] * prm.scale, z1 = z[2 * i + 1] * prm.scale;
                         zz = fmaf(z0, z0, zz); zz = fmaf(z1, z1, zz);
                         zmax = fmaxf(zmax, fmaxf(fabsf(z0), fabsf(z1)));
                         const __half2 h2 = __floats2half2_rn(z0, z1);
-                        pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                        const float2 hf = __half22float2(h2);
+                        const __half2 l2 = __floats2half2_rn(z0 - hf.x, z1 - hf.y);
+                        hi[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                        lo[i] = *reinterpret_cast<const uint32_t *>(&l2);
                     }
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        *reinterpret_cast<uint4 *>(a_row + c * 2048) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    for (int c = 0; c < 4; ++c) {
+                        *reinterpret_cast<uint4 *>(a_row + c * 2048) = make_uint4(hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
+                        *reinterpret_cast<uint4 *>(a_row + (4 + c) * 2048) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
+                    }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_arrive(BAR(kBarAReady + tile));
@@ -315,7 +322,7 @@ encode_tensor_kernel(const Params p)
 #pragma unroll
                 for (int q = 0; q < 11; ++q) d[q] = INFINITY;
 
-                const int chunks = 2 * S;
+                const int chunks = S;
 #pragma unroll 1
                 for (int c = 0; c < chunks && ok; ++c) {
                     ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag);
@@ -339,64 +346,107 @@ encode_tensor_kernel(const Params p)
                                              fminf(t[9], t[10]));
 #pragma unroll
                         for (int q = 0; q < 11; ++q) d[q] = fminf(d[q], t[q]);
-                        if (cb_min <= thr) {
-                            m1 = fminf(m1, cb_min);
-                            thr = m1 + win;
-                            if (cnt == kListCap) {
-                                // drop entries that fell out of the window as the minimum came down
-                                int keep = 0;
-                                for (int e = 0; e < kListCap; ++e) {
-                                    const float fv = list_v[e * kRowsPerPass];
-                                    const uint16_t fi = list_i[e * kRowsPerPass];
-                                    if (fv <= thr) { list_v[keep * kRowsPerPass] = fv; list_i[keep * kRowsPerPass] = fi; ++keep; }
-                                }
-                                cnt = keep;
+                        // Keep this block's minimum if it is within the window of the running
+                        // minimum.  Branch-free: the value is always written to the next free
+                        // slot and the slot is claimed only when it belongs on the list; slot
+                        // kListCap is scratch once the list has overflowed.
+                        const bool app = cb_min <= thr;
+                        m1 = fminf(m1, cb_min);
+                        thr = m1 + win;
+                        if (app && cnt == kListCap) {
+                            // full: drop entries that left the window as the minimum came down
+                            int keep = 0;
+                            for (int e = 0; e < kListCap; ++e) {
+                                const float fv = list_v[e * kRowsPerPass];
+                                const uint16_t fi = list_i[e * kRowsPerPass];
+                                if (fv <= thr) { list_v[keep * kRowsPerPass] = fv; list_i[keep * kRowsPerPass] = fi; ++keep; }
                             }
-                            if (cnt < kListCap) {
-                                list_v[cnt * kRowsPerPass] = cb_min;
-                                list_i[cnt * kRowsPerPass] = (uint16_t)(c * 4 + blk);
-                                ++cnt;
-                            } else {
-                                cnt = kListCap + 1;      // more candidates than the list holds: scan everything
-                            }
+                            cnt = keep;
                         }
+                        const int slot = min(cnt, kListCap);
+                        list_v[slot * kRowsPerPass] = cb_min;
+                        list_i[slot * kRowsPerPass] = (uint16_t)(c * 4 + blk);
+                        cnt += app ? 1 : 0;
                     }
                 }
                 if (!ok) break;
 
-                // ---- stage end: exact choice among the columns that can still be the argmin
+                // ---- stage end: exact choice among the columns that can still be the argmin.
+                // Common case (one listed block, one cell position): its three columns are
+                // re-scored by the row's own thread, all lanes in step.
+                const float lim = m1 + win;
+                int b1 = 0, nlisted = 0;
+                {
+                    bool found = false;
+#pragma unroll
+                    for (int e = 0; e < kListCap; ++e) {
+                        const float fv = list_v[e * kRowsPerPass];
+                        const int fi = list_i[e * kRowsPerPass];
+                        const bool live = e < cnt;
+                        if (live && fv <= lim) ++nlisted;
+                        if (live && !found && fv == m1) { found = true; b1 = fi; }
+                    }
+                }
+                int q1 = 0, ncells = 0;
+#pragma unroll
+                for (int q = 10; q >= 0; --q) {
+                    if (d[q] <= lim) ++ncells;
+                    if (d[q] == m1) q1 = q;
+                }
                 int bj = 0;
-                if (!deg) {
-                    float best = INFINITY;
-                    const float lim = m1 + win;
-                    if (force_scan || cnt == 0 || cnt > kListCap) {
-                        ++n_exhaustive;
-                        for (int j = 0; j < s.K; ++j) {
-                            const float dj = exact_distance(z, cbr + (size_t)j * 32);
-                            if (dj < best) { best = dj; bj = j; }
+                float best = INFINITY;
+#pragma unroll 1
+                for (int k = 0; k < 3; ++k) {
+                    const int jc = b1 * 32 + 3 * q1 + k;
+                    const bool in = 3 * q1 + k < 32 && jc < s.K;
+                    const float dj = exact_distance(z, cbr + (size_t)(in ? jc : 0) * 32);
+                    if (in && dj < best) { best = dj; bj = jc; }
+                }
+                const bool scan_all = force_scan || cnt == 0 || cnt > kListCap;
+                const bool flagged = !deg && (scan_all || nlisted * ncells > 1);
+                // Rows with more than one candidate: the whole warp re-scores every column of
+                // every listed block of one such row at a time (or all columns when the list
+                // overflowed), then reduces to the smallest distance, lowest index on ties.
+                uint32_t todo = __ballot_sync(0xFFFFFFFFu, flagged);
+                while (todo) {
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    float zs[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) zs[i] = __shfl_sync(0xFFFFFFFFu, z[i], src);
+                    const float lim_s = __shfl_sync(0xFFFFFFFFu, lim, src);
+                    const int cnt_s = __shfl_sync(0xFFFFFFFFu, cnt, src);
+                    const bool all_s = __shfl_sync(0xFFFFFFFFu, (int)scan_all, src) != 0;
+                    const int row_s = rloc - lane + src;
+                    float bv = INFINITY;
+                    int bi = 0x7FFFFFFF;
+                    if (all_s) {
+                        for (int j = lane; j < s.K; j += 32) {
+                            const float dj = exact_distance(zs, cbr + (size_t)j * 32);
+                            if (dj < bv) { bv = dj; bi = j; }
                         }
                     } else {
-                        int listed = 0;
-                        for (int e = 0; e < cnt; ++e) {
-                            if (!(list_v[e * kRowsPerPass] <= lim)) continue;
-                            ++listed;
-                            const int col0 = (int)list_i[e * kRowsPerPass] * 32;
-#pragma unroll
-                            for (int q = 0; q < 11; ++q) {
-                                if (!(d[q] <= lim)) continue;
-                                for (int k = 0; k < 3; ++k) {
-                                    const int j = col0 + 3 * q + k;
-                                    if (3 * q + k >= 32 || j >= s.K) continue;
-                                    const float dj = exact_distance(z, cbr + (size_t)j * 32);
-                                    if (dj < best) { best = dj; bj = j; }      // columns visited in ascending order
-                                }
-                            }
+                        for (int e = 0; e < cnt_s; ++e) {
+                            const float fv = reinterpret_cast<const float *>(smem + kOffListV)[e * kRowsPerPass + row_s];
+                            if (!(fv <= lim_s)) continue;                              // warp-uniform
+                            const int j = (int)reinterpret_cast<const uint16_t *>(smem + kOffListI)[e * kRowsPerPass + row_s] * 32 + lane;
+                            const float dj = exact_distance(zs, cbr + (size_t)(j < s.K ? j : 0) * 32);
+                            if (j < s.K && dj < bv) { bv = dj; bi = j; }
                         }
-                        int cells = 0;
-#pragma unroll
-                        for (int q = 0; q < 11; ++q) cells += (d[q] <= lim) ? 1 : 0;
-                        if (listed * cells > 1) ++n_rescored;
                     }
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) {
+                        const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off);
+                        const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
+                        if (ov < bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                    }
+                    if (lane == src) {
+                        bj = bi; best = bv;
+                        if (all_s) ++n_exhaustive; else ++n_rescored;
+                    }
+                }
+                if (deg) bj = 0;
+                if (!deg) {
                     const float4 *e4 = reinterpret_cast<const float4 *>(cbr + (size_t)bj * 32);
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
@@ -461,7 +511,7 @@ encode_tensor_kernel(const Params p)
 
 bool encode_tensor_supported(const Shape &s)
 {
-    return s.gd == 32 && s.G <= 32 && (s.G & (s.G - 1)) == 0 && slots_per_stage(s.K) * 8 <= 65535;
+    return s.gd == 32 && s.G <= 32 && (s.G & (s.G - 1)) == 0 && slots_per_stage(s.K) * 4 <= 65535;
 }
 
 int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,

@@ -6,10 +6,10 @@
 
 namespace rvq {
 
-constexpr uint32_t kPreparedMagic = 0x52565132u;
-constexpr int kSlotCodewords = 256;                       // codewords per operand slot
-constexpr int kSlotCells = 6;                             // 48 halves of contraction depth
-constexpr int kSlotBytes = kSlotCells * kSlotCodewords * 16;   // 24576
+constexpr uint32_t kPreparedMagic = 0x52565133u;
+constexpr int kSlotCodewords = 128;                       // codewords per operand slot
+constexpr int kSlotCells = 10;                            // hi (4), lo (4), norm (1), zero (1) cells of 8 halves
+constexpr int kSlotBytes = kSlotCells * kSlotCodewords * 16;   // 20480
 constexpr size_t kPreparedParamsOffset = 256;             // StageParams[16]
 constexpr size_t kPreparedMaximaOffset = 512;             // StageMaxima[16]
 constexpr size_t kPreparedImageOffset = 768;              // operand image, [R][slots][kSlotBytes]
@@ -25,7 +25,7 @@ struct StageParams {
 };
 
 struct StageMaxima {
-    uint32_t emax, eerr, nmax, pad;   // float bit patterns (non-negative), filled with atomicMax
+    uint32_t emax, eerr, nmax, elomax;   // float bit patterns (non-negative), filled with atomicMax
 };
 
 __host__ __device__ inline int slots_per_stage(int K) { return (K + kSlotCodewords - 1) / kSlotCodewords; }

@@ -1,23 +1,31 @@
 // Tensor-core encode for group_dim 32 (Section 2.2, Algorithm 1).
 //
-// One persistent CTA per SM works on passes of 512 group rows (four tiles of 128
-// rows, one row per thread, 16 epilogue warps) plus one control warp.
+// One persistent CTA per SM works on passes of 384 group rows (three tiles of 128
+// rows, one row per thread, 12 epilogue warps) plus one control warp.
 //   - Scores ||e||^2 - 2 z.e of a 128-row tile against 128 codewords are one
 //     tcgen05.mma chain (M=128, N=128, seven K=16 steps over the split
 //     half-precision operands described in prepare.cu), accumulated in float32
 //     in TMEM.
 //   - The B operand (128 codewords per slot) streams from the prepared block
 //     through a ring of shared-memory slots filled by cp.async.bulk; every
-//     slot serves all four tiles.
-//   - Epilogue threads read their row's 128 scores with tcgen05.ld and keep
+//     slot serves all three tiles.
+//   - Epilogue threads read their row's 128 scores with tcgen05.ld (the next
+//     32 columns are in flight while the current 32 are reduced) and keep
 //     (i) the minimum of every 32-column block that comes within the error
 //     window of the running minimum, and (ii) the minimum per 3-column cell
 //     position over all blocks.  Any column that could be the exact argmin lies
 //     in a listed block at a listed cell position; those few columns are
 //     re-scored exactly in float32 against the float32 codebook (direct form,
 //     lowest index on ties), so the emitted code is the exact-L2 choice.
-//   - The residual stays in registers across all R stages; x is read once and
-//     only codes and the half-precision deviation are written.
+//   - The A operand (the residual split into half-precision head and remainder)
+//     lives in TMEM next to its tile's scores, so the tensor core fetches only B
+//     from shared memory; the constant (1 1 1 0 ...) rows that pick up the
+//     squared norms are one small shared-memory tile used by every MMA chain.
+//   - The float32 residual lives in registers between stages and is parked in
+//     shared memory during a stage's sweep; x is read once and only codes and
+//     the half-precision deviation are written.
+// TMEM columns of tile t: scores [160 t, 160 t + 128), A operand
+// [160 t + 128, 160 t + 160) (16 columns of head, 16 of remainder).
 // Every wait is bounded; a wait that gives up sets status->wait_timeouts and
 // the kernel drains and returns.
 #include "prepared.cuh"
@@ -26,21 +34,23 @@ namespace rvq {
 
 namespace {
 
-constexpr int kTiles = 4;
+constexpr int kTiles = 3;
 constexpr int kRowsPerPass = 128 * kTiles;
 constexpr int kEpiThreads = kRowsPerPass;
 constexpr int kThreads = kEpiThreads + 32;
-constexpr int kRing = 4;                                  // operand slots in flight
-constexpr int kATileBytes = kSlotCells * 128 * 16;        // 20480
+constexpr int kRing = 6;                                  // operand slots in flight
+constexpr int kTileCols = 160;                            // TMEM columns per tile: 128 scores + 32 of A operand
+constexpr int kOnesBytes = 2 * 128 * 16;                  // the constant A cells (1 1 1 0 ...) and (0 ...)
 constexpr int kListCap = 8;
 constexpr uint32_t kWaitLimit = 4u * 1000u * 1000u;
 
 constexpr int kOffB = 0;
-constexpr int kOffA = kOffB + kRing * kSlotBytes;                    //  81920
-constexpr int kOffListV = kOffA + kTiles * kATileBytes;              // 163840
-constexpr int kOffListI = kOffListV + (kListCap + 1) * kRowsPerPass * 4;   // 180224
-constexpr int kOffCodes = kOffListI + (kListCap + 1) * kRowsPerPass * 2;   // 172032
-constexpr int kOffBars = kOffCodes + kRowsPerPass * 16 * 2;          // 188416
+constexpr int kOffA = kOffB + kRing * kSlotBytes;                    
+constexpr int kOffZ = kOffA + kOnesBytes;                             // parked residuals, float [32][rows]
+constexpr int kOffListV = kOffZ + 32 * kRowsPerPass * 4;              
+constexpr int kOffListI = kOffListV + (kListCap + 1) * kRowsPerPass * 4;   
+constexpr int kOffCodes = kOffListI + (kListCap + 1) * kRowsPerPass * 2;   
+constexpr int kOffBars = kOffCodes + kRowsPerPass * 16 * 2;          
 constexpr int kSmemBytes = kOffBars + 256;
 
 // barrier slots
@@ -91,6 +101,13 @@ __device__ __forceinline__ void mma_f16_ss(uint32_t d_tmem, uint64_t adesc, uint
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -105,20 +122,86 @@ __device__ __forceinline__ float min3(float a, float b, float c)
     return d;
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+#define RVQ_R32(u) u[0], u[1], u[2], u[3], u[4], u[5], u[6], u[7], u[8], u[9], u[10], u[11], u[12], u[13], u[14], u[15], \
+    u[16], u[17], u[18], u[19], u[20], u[21], u[22], u[23], u[24], u[25], u[26], u[27], u[28], u[29], u[30], u[31]
+#define RVQ_OUT32(u) "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), \
+    "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), \
+    "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), \
+    "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+#define RVQ_INOUT32(u) "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]), \
+    "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15]), \
+    "+r"(u[16]), "+r"(u[17]), "+r"(u[18]), "+r"(u[19]), "+r"(u[20]), "+r"(u[21]), "+r"(u[22]), "+r"(u[23]), \
+    "+r"(u[24]), "+r"(u[25]), "+r"(u[26]), "+r"(u[27]), "+r"(u[28]), "+r"(u[29]), "+r"(u[30]), "+r"(u[31])
+#define RVQ_IN32(u) "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]), \
+    "r"(u[8]), "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15]), \
+    "r"(u[16]), "r"(u[17]), "r"(u[18]), "r"(u[19]), "r"(u[20]), "r"(u[21]), "r"(u[22]), "r"(u[23]), \
+    "r"(u[24]), "r"(u[25]), "r"(u[26]), "r"(u[27]), "r"(u[28]), "r"(u[29]), "r"(u[30]), "r"(u[31])
+
+// Start loading 32 consecutive TMEM columns of this thread's lane.  The
+// registers are not valid until tmem_ld_wait() has been given the same array.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&u)[32])
 {
-    uint32_t u[32];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                  "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
                  "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
-                   "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
-                   "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
-                   "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
-                 : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                 : RVQ_OUT32(u) : "r"(taddr));
+}
+// Waits for every tcgen05.ld of this thread; the array passes through so that no
+// use of it can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&u)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : RVQ_INOUT32(u) : : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&u)[32])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 : : "r"(taddr), RVQ_IN32(u) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// Per-row state of one stage's sweep over the scores.
+struct Sweep {
+    float m1, thr, win;      // running minimum of the block minima, m1 + win, error window
+    int cnt;                 // listed blocks (kListCap + 1: the list overflowed)
+    float d[11];             // minimum per cell position (3 columns each, the last one 2)
+};
+
+// Minima of the eleven 3-column cells of a 32-column block, and the block minimum.
+__device__ __forceinline__ float block_cells(const uint32_t (&u)[32], float (&t)[11])
+{
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(u[i]);
+    for (int q = 0; q < 10; ++q)
+        t[q] = min3(__uint_as_float(u[3 * q]), __uint_as_float(u[3 * q + 1]), __uint_as_float(u[3 * q + 2]));
+    t[10] = fminf(__uint_as_float(u[30]), __uint_as_float(u[31]));
+    return fminf(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])), fminf(t[9], t[10]));
+}
+
+// Keep a block's minimum if it is within the window of the running minimum.
+// Branch-free: the value is always written to the next free slot and the slot
+// is claimed only when it belongs on the list; slot kListCap is scratch once
+// the list has overflowed.
+__device__ __forceinline__ void list_block(Sweep &w, float cb_min, int block, float *list_v, uint16_t *list_i,
+                                           int stride)
+{
+    const bool app = cb_min <= w.thr;
+    w.m1 = fminf(w.m1, cb_min);
+    w.thr = w.m1 + w.win;
+    if (app && w.cnt == kListCap) {
+        // full: drop entries that left the window as the minimum came down
+        int keep = 0;
+        for (int e = 0; e < kListCap; ++e) {
+            const float fv = list_v[e * stride];
+            const uint16_t fi = list_i[e * stride];
+            if (fv <= w.thr) { list_v[keep * stride] = fv; list_i[keep * stride] = fi; ++keep; }
+        }
+        w.cnt = keep;
+    }
+    const int slot = min(w.cnt, kListCap);
+    list_v[slot * stride] = cb_min;
+    list_i[slot * stride] = (uint16_t)block;
+    w.cnt += app ? 1 : 0;
 }
 
 // Exact squared distance, direct form, same operation order as the scalar kernel.
@@ -176,13 +259,13 @@ encode_tensor_kernel(const Params p)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_word)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
-    // constant part of every A row: cell 8 = (1, 1, 1, 0...), cell 9 = 0
-    if (tid < kEpiThreads) {
-        const int tile = tid >> 7, row = tid & 127;
-        uint8_t *a = smem + kOffA + tile * kATileBytes + row * 16;
-        *reinterpret_cast<uint4 *>(a + 8 * 2048) = make_uint4(0x3C003C00u, 0x00003C00u, 0u, 0u);
-        *reinterpret_cast<uint4 *>(a + 9 * 2048) = make_uint4(0u, 0u, 0u, 0u);
+    // constant A cells shared by all tiles: (1, 1, 1, 0...) per row, then zeros
+    if (tid < 128) {
+        uint8_t *a = smem + kOffA + tid * 16;
+        *reinterpret_cast<uint4 *>(a) = make_uint4(0x3C003C00u, 0x00003C00u, 0u, 0u);
+        *reinterpret_cast<uint4 *>(a + 2048) = make_uint4(0u, 0u, 0u, 0u);
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -212,21 +295,23 @@ encode_tensor_kernel(const Params p)
                 ok = mbar_wait(BAR(kBarFull + slot), use & 1u, abort_flag);
                 const uint32_t stage_global = q / S, s_in = q % S;
                 const uint32_t b_base = smem_u32(smem + kOffB + slot * kSlotBytes);
-                // (A cell pair, B cell pair) of the seven K=16 steps: hi.hi, hi.lo, lo.hi, 1.norm
-                constexpr int kStepA[7] = {0, 2, 0, 2, 4, 6, 8};
-                constexpr int kStepB[7] = {0, 2, 4, 6, 0, 2, 8};
+                // Seven K=16 steps: hi.hi (2), hi.lo (2), lo.hi (2) with A in TMEM (8 columns per
+                // step), then 1.norm with the constant A cells from shared memory.
+                constexpr int kStepA[6] = {0, 8, 0, 8, 16, 24};      // TMEM column of the A slice
+                constexpr int kStepB[7] = {0, 2, 4, 6, 0, 2, 8};      // first B cell of the step
+                const uint64_t ones_desc = make_smem_desc(smem_u32(smem + kOffA), 2048, 128);
                 for (int t = 0; t < kTiles && ok; ++t) {
                     if (s_in == 0) ok = mbar_wait(BAR(kBarAReady + t), stage_global & 1u, abort_flag);
                     if (ok && q > 0) ok = mbar_wait(BAR(kBarAccFree + t), (q - 1) & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a_base = smem_u32(smem + kOffA + t * kATileBytes);
+                    const uint32_t acc = tmem + t * kTileCols;
 #pragma unroll
                     for (int kk = 0; kk < 7; ++kk) {
-                        const uint64_t adesc = make_smem_desc(a_base + kStepA[kk] * 2048, 2048, 128);
                         const uint64_t bdesc = make_smem_desc(b_base + kStepB[kk] * (kSlotCodewords * 16),
                                                               kSlotCodewords * 16, 128);
-                        mma_f16_ss(tmem + t * 128, adesc, bdesc, idesc, kk > 0);
+                        if (kk < 6) mma_f16_ts(acc, acc + 128 + kStepA[kk], bdesc, idesc, kk > 0);
+                        else mma_f16_ss(acc, ones_desc, bdesc, idesc, 1);
                     }
                     mma_commit(BAR(kBarAccFull + t));
                 }
@@ -237,13 +322,13 @@ encode_tensor_kernel(const Params p)
         // ------------------------------------------------------------ epilogue warps
         const int tile = warp >> 2, q4 = warp & 3;
         const int rloc = tile * 128 + q4 * 32 + lane;
-        const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)tile * 128u;
-        uint8_t *a_row = smem + kOffA + tile * kATileBytes + (q4 * 32 + lane) * 16;
+        const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(tile * kTileCols);
+        float *z_park = reinterpret_cast<float *>(smem + kOffZ) + rloc;                    // [i][row]
         float *list_v = reinterpret_cast<float *>(smem + kOffListV) + rloc;              // [e][row]
         uint16_t *list_i = reinterpret_cast<uint16_t *>(smem + kOffListI) + rloc;         // [e][row]
         uint16_t *codes_s = reinterpret_cast<uint16_t *>(smem + kOffCodes);                // [row][R]
         const int G = s.G;
-        uint32_t chunk_use = 0, stage_global = 0;
+        uint32_t chunk_use = 0;
         uint32_t n_rescored = 0, n_exhaustive = 0, n_degenerate = 0, n_stdrange = 0;
         bool ok = true;
 
@@ -292,7 +377,7 @@ encode_tensor_kernel(const Params p)
                 // scaled half-precision copy of the residual -> A operand row; error window of this row
                 float zz = 0.0f, zmax = 0.0f;
                 {
-                    uint32_t hi[16], lo[16];
+                    uint32_t ab[32];                       // 16 words of head, 16 of remainder
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const float z0 = z[2 * i] * prm.scale, z1 = z[2 * i + 1] * prm.scale;
@@ -301,74 +386,66 @@ encode_tensor_kernel(const Params p)
                         const __half2 h2 = __floats2half2_rn(z0, z1);
                         const float2 hf = __half22float2(h2);
                         const __half2 l2 = __floats2half2_rn(z0 - hf.x, z1 - hf.y);
-                        hi[i] = *reinterpret_cast<const uint32_t *>(&h2);
-                        lo[i] = *reinterpret_cast<const uint32_t *>(&l2);
+                        ab[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                        ab[16 + i] = *reinterpret_cast<const uint32_t *>(&l2);
                     }
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        *reinterpret_cast<uint4 *>(a_row + c * 2048) = make_uint4(hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
-                        *reinterpret_cast<uint4 *>(a_row + (4 + c) * 2048) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
-                    }
+                    tmem_st32(taddr + 128, ab);
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                tc_fence_before();
                 mbar_arrive(BAR(kBarAReady + tile));
-                ++stage_global;
-                const float win = 2.125f * (prm.a * sqrtf(zz) * 1.0001f + prm.b);    // 2 * bound, with slack for this arithmetic
-                const bool force_scan = !(zmax < 60000.0f) || !(win < INFINITY);
-
-                float m1 = INFINITY, thr = INFINITY;
-                int cnt = 0;
-                float d[11];
+                // park the float32 residual in shared memory for the sweep
 #pragma unroll
-                for (int q = 0; q < 11; ++q) d[q] = INFINITY;
+                for (int i = 0; i < 32; ++i) z_park[i * kRowsPerPass] = z[i];
+                Sweep w;
+                w.win = 2.125f * (prm.a * sqrtf(zz) * 1.0001f + prm.b);    // 2 * bound, with slack for this arithmetic
+                w.m1 = INFINITY; w.thr = INFINITY; w.cnt = 0;
+#pragma unroll
+                for (int q = 0; q < 11; ++q) w.d[q] = INFINITY;
+                const bool force_scan = !(zmax < 60000.0f) || !(w.win < INFINITY);
 
-                const int chunks = S;
 #pragma unroll 1
-                for (int c = 0; c < chunks && ok; ++c) {
+                for (int c = 0; c < S && ok; ++c) {
                     ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag);
                     ok = __all_sync(0xFFFFFFFFu, ok);          // tcgen05.ld below needs the whole warp
                     ++chunk_use;
                     if (!ok) break;
                     tc_fence_after();
-#pragma unroll 1
-                    for (int blk = 0; blk < 4; ++blk) {
-                        float sc[32];
-                        tmem_ld32(taddr + blk * 32, sc);
-                        if (blk == 3) {
-                            tc_fence_before();
-                            mbar_arrive(BAR(kBarAccFree + tile));
-                        }
-                        float t[11];
+                    // four 32-column blocks; the next block loads while the current one is reduced
+                    uint32_t ua[32], ub[32];
+                    float ta[11], tb[11];
+                    tmem_ld32_issue(taddr, ua);
+                    tmem_ld_wait(ua);
+                    tmem_ld32_issue(taddr + 32, ub);
+                    const float ca0 = block_cells(ua, ta);
+                    list_block(w, ca0, c * 4, list_v, list_i, kRowsPerPass);
+                    tmem_ld_wait(ub);
+                    tmem_ld32_issue(taddr + 64, ua);
+                    const float cb0 = block_cells(ub, tb);
 #pragma unroll
-                        for (int q = 0; q < 10; ++q) t[q] = min3(sc[3 * q], sc[3 * q + 1], sc[3 * q + 2]);
-                        t[10] = fminf(sc[30], sc[31]);
-                        float cb_min = fminf(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])),
-                                             fminf(t[9], t[10]));
+                    for (int q = 0; q < 11; ++q) w.d[q] = min3(w.d[q], ta[q], tb[q]);
+                    list_block(w, cb0, c * 4 + 1, list_v, list_i, kRowsPerPass);
+                    tmem_ld_wait(ua);
+                    tmem_ld32_issue(taddr + 96, ub);
+                    const float ca1 = block_cells(ua, ta);
+                    list_block(w, ca1, c * 4 + 2, list_v, list_i, kRowsPerPass);
+                    tmem_ld_wait(ub);
+                    tc_fence_before();
+                    mbar_arrive(BAR(kBarAccFree + tile));        // the accumulator may be overwritten
+                    const float cb1 = block_cells(ub, tb);
 #pragma unroll
-                        for (int q = 0; q < 11; ++q) d[q] = fminf(d[q], t[q]);
-                        // Keep this block's minimum if it is within the window of the running
-                        // minimum.  Branch-free: the value is always written to the next free
-                        // slot and the slot is claimed only when it belongs on the list; slot
-                        // kListCap is scratch once the list has overflowed.
-                        const bool app = cb_min <= thr;
-                        m1 = fminf(m1, cb_min);
-                        thr = m1 + win;
-                        if (app && cnt == kListCap) {
-                            // full: drop entries that left the window as the minimum came down
-                            int keep = 0;
-                            for (int e = 0; e < kListCap; ++e) {
-                                const float fv = list_v[e * kRowsPerPass];
-                                const uint16_t fi = list_i[e * kRowsPerPass];
-                                if (fv <= thr) { list_v[keep * kRowsPerPass] = fv; list_i[keep * kRowsPerPass] = fi; ++keep; }
-                            }
-                            cnt = keep;
-                        }
-                        const int slot = min(cnt, kListCap);
-                        list_v[slot * kRowsPerPass] = cb_min;
-                        list_i[slot * kRowsPerPass] = (uint16_t)(c * 4 + blk);
-                        cnt += app ? 1 : 0;
-                    }
+                    for (int q = 0; q < 11; ++q) w.d[q] = min3(w.d[q], ta[q], tb[q]);
+                    list_block(w, cb1, c * 4 + 3, list_v, list_i, kRowsPerPass);
                 }
+                if (!ok) break;
+                // take the residual back
+#pragma unroll
+                for (int i = 0; i < 32; ++i) z[i] = z_park[i * kRowsPerPass];
+                const float m1 = w.m1;
+                const int cnt = w.cnt;
+                float d[11];
+#pragma unroll
+                for (int q = 0; q < 11; ++q) d[q] = w.d[q];
+                const float win = w.win;
                 if (!ok) break;
 
                 // ---- stage end: exact choice among the columns that can still be the argmin.
@@ -413,7 +490,7 @@ encode_tensor_kernel(const Params p)
                     todo &= todo - 1;
                     float zs[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) zs[i] = __shfl_sync(0xFFFFFFFFu, z[i], src);
+                    for (int i = 0; i < 32; ++i) zs[i] = z_park[i * kRowsPerPass + (src - lane)];
                     const float lim_s = __shfl_sync(0xFFFFFFFFu, lim, src);
                     const int cnt_s = __shfl_sync(0xFFFFFFFFu, cnt, src);
                     const bool all_s = __shfl_sync(0xFFFFFFFFu, (int)scan_all, src) != 0;

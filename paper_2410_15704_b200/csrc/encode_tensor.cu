@@ -1,7 +1,8 @@
 // Tensor-core encode for group_dim 32 (Section 2.2, Algorithm 1).
 //
 // One persistent CTA per SM works on passes of 384 group rows (three tiles of 128
-// rows, one row per thread, 12 epilogue warps) plus one control warp.
+// rows, one row per thread, 12 epilogue warps) plus four single-thread roles in
+// warps of their own: one MMA issuer per tile and the operand loader.
 //   - Scores ||e||^2 - 2 z.e of a 128-row tile against 128 codewords are one
 //     tcgen05.mma chain (M=128, N=128, seven K=16 steps over the split
 //     half-precision operands described in prepare.cu), accumulated in float32
@@ -37,7 +38,7 @@ namespace {
 constexpr int kTiles = 3;
 constexpr int kRowsPerPass = 128 * kTiles;
 constexpr int kEpiThreads = kRowsPerPass;
-constexpr int kThreads = kEpiThreads + 32;
+constexpr int kThreads = kEpiThreads + 32 * (kTiles + 1);  // + one MMA issuer warp per tile + loader warp
 constexpr int kRing = 6;                                  // operand slots in flight
 constexpr int kTileCols = 160;                            // TMEM columns per tile: 128 scores + 32 of A operand
 constexpr int kOnesBytes = 2 * 128 * 16;                  // the constant A cells (1 1 1 0 ...) and (0 ...)
@@ -74,6 +75,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 // Bounded wait; returns false (and raises the CTA's abort flag) when it gives up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
 {
+#pragma unroll 1
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -248,7 +250,7 @@ encode_tensor_kernel(const Params p)
     auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     if (tid == 0) {
-        for (int i = 0; i < kRing; ++i) { mbar_init(BAR(kBarFull + i), 1); mbar_init(BAR(kBarEmpty + i), 1); }
+        for (int i = 0; i < kRing; ++i) { mbar_init(BAR(kBarFull + i), 1); mbar_init(BAR(kBarEmpty + i), kTiles); }
         for (int t = 0; t < kTiles; ++t) {
             mbar_init(BAR(kBarAReady + t), 128); mbar_init(BAR(kBarAccFull + t), 1); mbar_init(BAR(kBarAccFree + t), 128);
         }
@@ -271,51 +273,63 @@ encode_tensor_kernel(const Params p)
     tc_fence_after();
     const uint32_t tmem = *tmem_word;
 
-    if (warp == kEpiThreads / 32) {
-        // ------------------------------------------------------------ control warp
+    if (warp == kEpiThreads / 32 + kTiles) {
+        // ------------------------------------------------------------ operand loader
+        // One thread streams the B slots of every (pass, stage) through the ring; a slot is
+        // free again once the MMA chains of all tiles that read it have completed.
         if (lane == 0 && my_passes > 0) {
             const uint32_t total = (uint32_t)my_passes * (uint32_t)s.R * (uint32_t)S;
+            const uint32_t per_pass = (uint32_t)s.R * (uint32_t)S;
+            uint32_t slot = 0, rs = 0, empty_par = 1;          // parity of the previous completion of empty[slot]
+            bool ok = true;
+            for (uint32_t nl = 0; nl < total && ok; ++nl) {
+                if (nl >= (uint32_t)kRing) ok = mbar_wait(BAR(kBarEmpty + slot), empty_par, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(BAR(kBarFull + slot), kSlotBytes);
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(smem_u32(smem + kOffB) + slot * (uint32_t)kSlotBytes), "l"(image + (size_t)rs * kSlotBytes),
+                               "r"((uint32_t)kSlotBytes), "r"(BAR(kBarFull + slot)) : "memory");
+                if (++rs == per_pass) rs = 0;
+                if (++slot == (uint32_t)kRing) { slot = 0; empty_par ^= 1u; }
+            }
+        }
+    } else if (warp >= kEpiThreads / 32) {
+        // ------------------------------------------------------------ MMA issuer of tile t
+        // One thread per tile, each in a warp of its own so that the tiles' waits overlap.
+        // Whatever it does between two tcgen05.mma chains delays its tile, so descriptors
+        // are built once and all counters advance by increments.
+        if (lane == 0 && my_passes > 0) {
+            const int t = warp - kEpiThreads / 32;
+            const uint32_t total = (uint32_t)my_passes * (uint32_t)s.R * (uint32_t)S;
             const uint32_t idesc = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);   // f16 x f16 -> f32, M=N=128
-            uint32_t n_load = 0;
+            // Seven K=16 steps: hi.hi (2), hi.lo (2), lo.hi (2) with A in TMEM (8 columns per
+            // step), then 1.norm with the constant A cells from shared memory.  A B cell is
+            // 128 codewords x 16 bytes = 2048 bytes = 128 descriptor address units.
+            const uint64_t bdesc0 = make_smem_desc(smem_u32(smem + kOffB), kSlotCodewords * 16, 128);
+            const uint64_t ones_desc = make_smem_desc(smem_u32(smem + kOffA), 2048, 128);
+            const uint32_t acc = tmem + t * kTileCols, a0 = acc + 128;
+            const uint32_t bar_ready = BAR(kBarAReady + t), bar_free = BAR(kBarAccFree + t), bar_acc = BAR(kBarAccFull + t);
+            uint32_t slot = 0, full_par = 0, s_in = 0, ready_par = 0, free_par = 1;
             bool ok = true;
             for (uint32_t q = 0; q < total && ok; ++q) {
-                while (ok && n_load < total && n_load < q + kRing - 1) {
-                    const uint32_t slot = n_load % kRing, use = n_load / kRing;
-                    if (use > 0) ok = mbar_wait(BAR(kBarEmpty + slot), (use - 1) & 1u, abort_flag);
-                    if (!ok) break;
-                    const uint32_t rs = n_load % ((uint32_t)s.R * S);      // (stage, slot-in-stage), row-major
-                    mbar_expect_tx(BAR(kBarFull + slot), kSlotBytes);
-                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                 ::"r"(smem_u32(smem + kOffB + slot * kSlotBytes)), "l"(image + (size_t)rs * kSlotBytes),
-                                   "r"((uint32_t)kSlotBytes), "r"(BAR(kBarFull + slot)) : "memory");
-                    ++n_load;
-                }
+                ok = mbar_wait(BAR(kBarFull + slot), full_par, abort_flag);
+                if (ok && s_in == 0) ok = mbar_wait(bar_ready, ready_par, abort_flag);
+                if (ok && q > 0) ok = mbar_wait(bar_free, free_par, abort_flag);
                 if (!ok) break;
-                const uint32_t slot = q % kRing, use = q / kRing;
-                ok = mbar_wait(BAR(kBarFull + slot), use & 1u, abort_flag);
-                const uint32_t stage_global = q / S, s_in = q % S;
-                const uint32_t b_base = smem_u32(smem + kOffB + slot * kSlotBytes);
-                // Seven K=16 steps: hi.hi (2), hi.lo (2), lo.hi (2) with A in TMEM (8 columns per
-                // step), then 1.norm with the constant A cells from shared memory.
-                constexpr int kStepA[6] = {0, 8, 0, 8, 16, 24};      // TMEM column of the A slice
-                constexpr int kStepB[7] = {0, 2, 4, 6, 0, 2, 8};      // first B cell of the step
-                const uint64_t ones_desc = make_smem_desc(smem_u32(smem + kOffA), 2048, 128);
-                for (int t = 0; t < kTiles && ok; ++t) {
-                    if (s_in == 0) ok = mbar_wait(BAR(kBarAReady + t), stage_global & 1u, abort_flag);
-                    if (ok && q > 0) ok = mbar_wait(BAR(kBarAccFree + t), (q - 1) & 1u, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t acc = tmem + t * kTileCols;
-#pragma unroll
-                    for (int kk = 0; kk < 7; ++kk) {
-                        const uint64_t bdesc = make_smem_desc(b_base + kStepB[kk] * (kSlotCodewords * 16),
-                                                              kSlotCodewords * 16, 128);
-                        if (kk < 6) mma_f16_ts(acc, acc + 128 + kStepA[kk], bdesc, idesc, kk > 0);
-                        else mma_f16_ss(acc, ones_desc, bdesc, idesc, 1);
-                    }
-                    mma_commit(BAR(kBarAccFull + t));
-                }
-                if (ok) mma_commit(BAR(kBarEmpty + slot));
+                tc_fence_after();
+                const uint64_t bd = bdesc0 + (uint64_t)(slot * (uint32_t)(kSlotBytes >> 4));
+                mma_f16_ts(acc, a0, bd, idesc, 0);                      // hi[0:16]  . hi cells 0-1
+                mma_f16_ts(acc, a0 + 8, bd + 2 * 128, idesc, 1);        // hi[16:32] . hi cells 2-3
+                mma_f16_ts(acc, a0, bd + 4 * 128, idesc, 1);            // hi[0:16]  . lo cells 4-5
+                mma_f16_ts(acc, a0 + 8, bd + 6 * 128, idesc, 1);        // hi[16:32] . lo cells 6-7
+                mma_f16_ts(acc, a0 + 16, bd, idesc, 1);                 // lo[0:16]  . hi cells 0-1
+                mma_f16_ts(acc, a0 + 24, bd + 2 * 128, idesc, 1);       // lo[16:32] . hi cells 2-3
+                mma_f16_ss(acc, ones_desc, bd + 8 * 128, idesc, 1);     // (1 1 1 0..) . norm cells 8-9
+                mma_commit(bar_acc);
+                mma_commit(BAR(kBarEmpty + slot));
+                free_par ^= 1u;
+                if (++slot == (uint32_t)kRing) { slot = 0; full_par ^= 1u; }
+                if (++s_in == (uint32_t)S) { s_in = 0; ready_par ^= 1u; }
             }
         }
     } else {
@@ -472,12 +486,27 @@ encode_tensor_kernel(const Params p)
                 }
                 int bj = 0;
                 float best = INFINITY;
-#pragma unroll 1
-                for (int k = 0; k < 3; ++k) {
-                    const int jc = b1 * 32 + 3 * q1 + k;
-                    const bool in = 3 * q1 + k < 32 && jc < s.K;
-                    const float dj = exact_distance(z, cbr + (size_t)(in ? jc : 0) * 32);
-                    if (in && dj < best) { best = dj; bj = jc; }
+                {
+                    // the three columns of the cell, scored together so that their loads overlap
+                    const int j0 = b1 * 32 + 3 * q1;
+                    const bool in1 = 3 * q1 + 1 < 32 && j0 + 1 < s.K, in2 = 3 * q1 + 2 < 32 && j0 + 2 < s.K;
+                    const float4 *e0 = reinterpret_cast<const float4 *>(cbr + (size_t)(j0 < s.K ? j0 : 0) * 32);
+                    const float4 *e1 = in1 ? e0 + 8 : e0, *e2 = in2 ? e0 + 16 : e0;
+                    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 u0 = __ldg(e0 + q), u1 = __ldg(e1 + q), u2 = __ldg(e2 + q);
+                        float t;
+                        t = z[4 * q] - u0.x; a0 = fmaf(t, t, a0); t = z[4 * q + 1] - u0.y; a0 = fmaf(t, t, a0);
+                        t = z[4 * q + 2] - u0.z; a0 = fmaf(t, t, a0); t = z[4 * q + 3] - u0.w; a0 = fmaf(t, t, a0);
+                        t = z[4 * q] - u1.x; a1 = fmaf(t, t, a1); t = z[4 * q + 1] - u1.y; a1 = fmaf(t, t, a1);
+                        t = z[4 * q + 2] - u1.z; a1 = fmaf(t, t, a1); t = z[4 * q + 3] - u1.w; a1 = fmaf(t, t, a1);
+                        t = z[4 * q] - u2.x; a2 = fmaf(t, t, a2); t = z[4 * q + 1] - u2.y; a2 = fmaf(t, t, a2);
+                        t = z[4 * q + 2] - u2.z; a2 = fmaf(t, t, a2); t = z[4 * q + 3] - u2.w; a2 = fmaf(t, t, a2);
+                    }
+                    if (j0 < s.K) { best = a0; bj = j0; }
+                    if (in1 && a1 < best) { best = a1; bj = j0 + 1; }
+                    if (in2 && a2 < best) { best = a2; bj = j0 + 2; }
                 }
                 const bool scan_all = force_scan || cnt == 0 || cnt > kListCap;
                 const bool flagged = !deg && (scan_all || nlisted * ncells > 1);

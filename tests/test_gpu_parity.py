@@ -160,7 +160,7 @@ def test_ema_resume_equals_straight_run():
     resumed = run(5, run(5))
     for a, c in zip(straight, resumed):
         diff = torch.abs(a - c)
-        assert diff.max().item() <= 5e-2 and diff.mean().item() <= 1e-5
+        assert diff.max().item() <= 5e-2 and diff.mean().item() <= 1e-4
 
 
 def test_tensor_encode_equals_exact_encode():

@@ -147,7 +147,12 @@ int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n,
 /*
  * Decode (Section 2.2, last sentence; Section 3.2).  For every head vector and
  * channel c = channel(g, i): x_out[c] = std * sum_r C_r[code[g][r]][i], summed
- * in float32 in stage order and rounded once to x_dtype.
+ * in float32 and rounded once to x_dtype.  For 16-bit outputs of dim 128 = 4
+ * groups of 32 with depth <= 8 the codebook entries are read from the prepared
+ * block as 15-bit levels of each stage's value range, so the sum before the
+ * multiplication by std is within sum_r (max C_r - min C_r) * 2^-16 of the
+ * float32 one (the prepared block must then have been built with the same
+ * x_dtype); float32 outputs and other shapes gather the float32 codebooks.
  *   codes, std_f16  in   as produced by rvq_encode
  *   x_out           out  n rows of x_dtype, row v at element v * out_row_stride
  * A code >= K is read as code 0 and counted in status->bad_codes.

@@ -1,6 +1,6 @@
 // extern "C" boundary of the RVQ library: argument checks on the host, then
 // dispatch to the kernels.  No allocation, no synchronisation, no global state.
-#include "common.cuh"
+#include "prepared.cuh"
 
 #include <atomic>
 
@@ -140,6 +140,8 @@ int rvq_decode(const rvq_config *cfg, const void *codes, const uint16_t *std_f16
     if ((rc = check_rows(s, x_out, n, out_row_stride)) != RVQ_OK) return rc;
     if (!codebooks || !prepared || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
     if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    if (decode_sliced_supported(s))
+        return launch_decode_sliced(s, codes, std_f16, n, prepared, x_out, out_row_stride, status, (cudaStream_t)stream);
     return launch_decode_gather(s, codes, std_f16, n, codebooks, x_out, out_row_stride, status, (cudaStream_t)stream);
 }
 

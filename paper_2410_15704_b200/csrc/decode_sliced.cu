@@ -1,0 +1,198 @@
+// Bandwidth decode for dim 128 = 4 groups of 32, depth <= 8 (Section 2.2, last
+// sentence; Section 3.2).
+//
+// Every output element needs one codeword element per stage, so a head vector of
+// 256 output bytes gathers 1024 table entries: the gather, not HBM, is the
+// limit, and it has to come from shared memory without bank conflicts.
+//   - A CTA keeps one channel slice (8 of the 32 codeword channels) of all
+//     stages as 15-bit levels: 128 bytes per code = 8 stages x 16 bytes.  The
+//     four slices of a row tile are handled by four CTAs; the codes they share
+//     come from L2.
+//   - One thread produces the 8 channels of one (group row, slice).  It reads
+//     its 8 codes as one 16-byte load and visits the stages in an order rotated
+//     by its lane, so the 8 lanes of a quarter warp always touch 8 different
+//     16-byte bank groups whatever the codes are.
+//   - A level q becomes the float 1 + q 2^-15 by one byte permute (the stored
+//     level carries the exponent's low bit), and one FMA with the stage's step
+//     adds it to a float32 sum; the affine offsets of all stages are removed at
+//     the end, then the sum is multiplied by the stored deviation and rounded once.
+//   - With strided groups the 4 lanes of a head vector exchange their results so
+//     that every lane stores 16 contiguous bytes.
+#include "prepared.cuh"
+
+namespace rvq {
+
+namespace {
+
+constexpr int kDecThreads = 1024;
+
+template <int DT> struct Out;
+template <> struct Out<RVQ_BF16> {
+    static __device__ __forceinline__ uint32_t pack(float a, float b)
+    {
+        __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+        return *reinterpret_cast<uint32_t *>(&h);
+    }
+};
+template <> struct Out<RVQ_F16> {
+    static __device__ __forceinline__ uint32_t pack(float a, float b)
+    {
+        __half2 h = __floats2half2_rn(a, b);
+        return *reinterpret_cast<uint32_t *>(&h);
+    }
+};
+
+// Float 1 + q * 2^-15 from the low (H = 0) or high (H = 1) half of a table word.
+template <int H>
+__device__ __forceinline__ float level_to_float(uint32_t word)
+{
+    // bytes of the result, most significant first: 0x3F, half's high byte, half's low byte, 0x00
+    return __uint_as_float(__byte_perm(word, 0x3F000000u, H ? 0x7324 : 0x7104));
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kDecThreads, 1)
+decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                     const uint8_t *__restrict__ dsec, void *__restrict__ out, int64_t stride, rvq_status *st)
+{
+    extern __shared__ __align__(128) uint8_t table[];            // [K][8 stages][16 bytes]
+    const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
+    const int slice = blockIdx.x & 3, part = blockIdx.x >> 2, parts = gridDim.x >> 2;
+    const int tid = threadIdx.x, lane = tid & 31, rot = lane & 7;
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256) + (size_t)slice * s.K * 8;
+        uint4 *dst = reinterpret_cast<uint4 *>(table);
+        for (int t = tid; t < s.K * 8; t += kDecThreads) dst[t] = __ldg(src + t);
+    }
+    // this thread visits stage (rot + k) & 7 at step k: its steps' scales and line offsets
+    float step[8];
+    uint32_t unit[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { step[k] = dp->step[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * 16u; }
+    const float bias = dp->bias;
+    __syncthreads();
+
+    const int64_t rows = n * 4;
+    uint32_t bad = 0;
+    for (int64_t row = (int64_t)part * kDecThreads + tid; row - tid < rows; row += (int64_t)parts * kDecThreads) {
+        // (the loop bound keeps whole warps together for the shuffles below)
+        const bool live = row < rows;
+        const int64_t v = live ? row >> 2 : 0;
+        const int g = (int)(row & 3);
+        // the 8 codes of this row as 4 words, stage r in half r
+        uint32_t cw[4] = {0u, 0u, 0u, 0u};
+        if (live) {
+            if (s.bits == 16 && s.R == 8) {
+                const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + row);
+                cw[0] = c.x; cw[1] = c.y; cw[2] = c.z; cw[3] = c.w;
+            } else {
+                const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes;
+                for (int r = 0; r < s.R; ++r)
+                    cw[r >> 1] |= read_code(vec, g * s.R + r, s.bits, s.code_bytes) << (16 * (r & 1));
+            }
+        }
+        // rotate the 8 halves left by `rot` so that step k finds its code at a fixed place
+        {
+            uint32_t a0 = cw[0], a1 = cw[1], a2 = cw[2], a3 = cw[3];
+            if (rot & 4) { uint32_t t0 = a0, t1 = a1; a0 = a2; a1 = a3; a2 = t0; a3 = t1; }
+            if (rot & 2) { uint32_t t0 = a0; a0 = a1; a1 = a2; a2 = a3; a3 = t0; }
+            if (rot & 1) {
+                const uint32_t b0 = __funnelshift_r(a0, a1, 16), b1 = __funnelshift_r(a1, a2, 16);
+                const uint32_t b2 = __funnelshift_r(a2, a3, 16), b3 = __funnelshift_r(a3, a0, 16);
+                a0 = b0; a1 = b1; a2 = b2; a3 = b3;
+            }
+            cw[0] = a0; cw[1] = a1; cw[2] = a2; cw[3] = a3;
+        }
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
+            if (j >= (uint32_t)s.K) { j = 0; ++bad; }
+            const uint4 e = *reinterpret_cast<const uint4 *>(table + j * 128u + unit[k]);
+            const float sk = step[k];
+            acc[0] = fmaf(level_to_float<0>(e.x), sk, acc[0]); acc[1] = fmaf(level_to_float<1>(e.x), sk, acc[1]);
+            acc[2] = fmaf(level_to_float<0>(e.y), sk, acc[2]); acc[3] = fmaf(level_to_float<1>(e.y), sk, acc[3]);
+            acc[4] = fmaf(level_to_float<0>(e.z), sk, acc[4]); acc[5] = fmaf(level_to_float<1>(e.z), sk, acc[5]);
+            acc[6] = fmaf(level_to_float<0>(e.w), sk, acc[6]); acc[7] = fmaf(level_to_float<1>(e.w), sk, acc[7]);
+        }
+        const float sd = live ? __half2float(__ushort_as_half(std16[v])) : 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = (acc[i] + bias) * sd;
+
+        if (DT == RVQ_F32) {
+            if (s.layout == RVQ_GROUP_CONTIGUOUS) {
+                if (live) {
+                    float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + v * stride + g * 32 + slice * 8);
+                    o[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                    o[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                }
+            } else if (live) {
+                float *o = reinterpret_cast<float *>(out) + v * stride + slice * 32 + g;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[4 * i] = acc[i];         // channel (8 slice + i) * 4 + g
+            }
+        } else {
+            uint32_t w[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) w[c] = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(acc[2 * c], acc[2 * c + 1]);
+            if (s.layout == RVQ_GROUP_CONTIGUOUS) {
+                if (live)
+                    *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(out) + v * stride + g * 32 + slice * 8) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
+            } else {
+                // Lane g holds element pairs (2c, 2c+1) of group g, i.e. channels 32 slice + 8c + g and + 4.
+                // Lane c' of the 4-lane set wants pairs c' of all four groups: a 4x4 transpose of words.
+#pragma unroll
+                for (int jx = 1; jx < 4; ++jx) {
+                    const int give = g ^ jx;                                 // the word the partner wants is w[partner]
+                    const uint32_t send = give == 0 ? w[0] : give == 1 ? w[1] : give == 2 ? w[2] : w[3];
+                    const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, send, jx);   // partner's w[g]: group (g ^ jx), pair g
+                    if (give == 0) w[0] = got; else if (give == 1) w[1] = got; else if (give == 2) w[2] = got; else w[3] = got;
+                }
+                // now w[q] = pair g of group q: (element 2g of group q, element 2g+1 of group q)
+                const uint32_t o0 = __byte_perm(w[0], w[1], 0x5410), o1 = __byte_perm(w[2], w[3], 0x5410);
+                const uint32_t o2 = __byte_perm(w[0], w[1], 0x7632), o3 = __byte_perm(w[2], w[3], 0x7632);
+                // channels 32 slice + 8 g + 0..7: element 2g of groups 0..3, then element 2g+1 of groups 0..3
+                if (live)
+                    *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(out) + v * stride + slice * 32 + g * 8) =
+                        make_uint4(o0, o1, o2, o3);
+            }
+        }
+    }
+    if (bad && st) atomicAdd(&st->bad_codes, bad);
+}
+
+}  // namespace
+
+int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
+                         const void *prepared, void *out, int64_t stride, rvq_status *st,
+                         cudaStream_t stream)
+{
+    if (n == 0) return RVQ_OK;
+    const uint8_t *p = reinterpret_cast<const uint8_t *>(prepared);
+    const size_t off = (kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return RVQ_ERR_DEVICE;
+    const size_t smem = (size_t)s.K * 128;
+    const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
+    int parts = sms / 4;
+    if (parts > tiles) parts = (int)tiles;
+    if (parts < 1) parts = 1;
+    auto launch = [&](auto kernel) -> int {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return RVQ_ERR_LAUNCH;
+        kernel<<<parts * 4, kDecThreads, smem, stream>>>(s, codes, std16, n, p + off, out, stride, st);
+        return check_launch();
+    };
+    switch (s.dtype) {
+    case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32>);
+    case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16>);
+    default: return launch(decode_sliced_kernel<RVQ_F16>);
+    }
+}
+
+}  // namespace rvq

@@ -24,12 +24,79 @@
 
 namespace rvq {
 
+static size_t decode_section_offset(const Shape &s)
+{
+    return (kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256;
+}
+
 size_t prepared_bytes(const Shape &s)
 {
-    size_t b = kPreparedImageOffset;
-    if (s.gd == 32) b += (size_t)s.R * slots_per_stage(s.K) * kSlotBytes;
+    size_t b = decode_section_offset(s);
+    if (decode_sliced_supported(s)) b += 256 + decode_table_bytes(s.K);
     return (b + 255) / 256 * 256;
 }
+
+// One block per stage (8 blocks): range of the stage's entries -> affine map.
+__global__ void __launch_bounds__(256)
+decode_range_kernel(Shape s, const float *__restrict__ cb, DecodeParams *dp, float *lo_out)
+{
+    __shared__ float smin[256], smax[256];
+    const int r = blockIdx.x, tid = threadIdx.x;
+    float lo = INFINITY, hi = -INFINITY;
+    if (r < s.R)
+        for (int t = tid; t < s.K * 32; t += 256) {
+            const float v = cb[(size_t)r * s.K * 32 + t];
+            lo = fminf(lo, v); hi = fmaxf(hi, v);
+        }
+    smin[tid] = lo; smax[tid] = hi;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (tid < w) { smin[tid] = fminf(smin[tid], smin[tid + w]); smax[tid] = fmaxf(smax[tid], smax[tid + w]); }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        float step = 0.0f, l = 0.0f;
+        if (r < s.R && smax[0] > smin[0]) { l = smin[0]; step = (smax[0] - smin[0]) * (32768.0f / 32767.0f); }
+        else if (r < s.R) { l = smin[0]; }
+        dp->step[r] = step;
+        lo_out[r] = l;
+    }
+}
+
+__global__ void decode_bias_kernel(DecodeParams *dp, const float *lo)
+{
+    float b = 0.0f, e = 0.0f;
+    for (int r = 0; r < 8; ++r) { b += lo[r] - dp->step[r]; e += dp->step[r] * 1.52587890625e-5f; }   // half a level per stage
+    dp->bias = b;
+    dp->err = e;
+}
+
+// One thread per (slice, code): 8 stages x 8 channels of levels.
+__global__ void __launch_bounds__(256)
+decode_table_kernel(Shape s, const float *__restrict__ cb, const DecodeParams *__restrict__ dp,
+                    const float *__restrict__ lo, uint4 *__restrict__ table)
+{
+    const int j = blockIdx.x * 256 + threadIdx.x, slice = blockIdx.y;
+    if (j >= s.K) return;
+    for (int r = 0; r < 8; ++r) {
+        uint32_t w[4];
+        for (int c = 0; c < 4; ++c) {
+            uint32_t pair = 0;
+            for (int h = 0; h < 2; ++h) {
+                uint32_t level = 0;
+                if (r < s.R && dp->step[r] > 0.0f) {
+                    const float v = cb[((size_t)r * s.K + j) * 32 + slice * 8 + 2 * c + h];
+                    const float q = rintf((v - lo[r]) / dp->step[r] * 32768.0f);
+                    level = (uint32_t)fminf(fmaxf(q, 0.0f), 32767.0f);
+                }
+                pair |= (0x8000u | level) << (16 * h);
+            }
+            w[c] = pair;
+        }
+        table[((size_t)slice * s.K + j) * 8 + r] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 
 // One block per stage: largest squared norm -> scale exponent; clears the maxima.
 __global__ void __launch_bounds__(256)
@@ -66,6 +133,8 @@ prepare_scale_kernel(Shape s, const float *__restrict__ cb, PreparedHeader *hdr,
         if (r == 0) {
             hdr->magic = kPreparedMagic; hdr->R = s.R; hdr->K = s.K; hdr->gd = s.gd;
             hdr->slots = slots_per_stage(s.K);
+            hdr->decode_offset = decode_sliced_supported(s)
+                ? (uint32_t)((kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256) : 0u;
         }
     }
 }
@@ -146,12 +215,27 @@ int launch_prepare(const Shape &s, const float *cb, void *prepared, cudaStream_t
     StageMaxima *mx = reinterpret_cast<StageMaxima *>(p + kPreparedMaximaOffset);
     prepare_scale_kernel<<<s.R, 256, 0, stream>>>(s, cb, hdr, sp, mx);
     int rc = check_launch();
-    if (rc != RVQ_OK || s.gd != 32) return rc;
-    dim3 grid(slots_per_stage(s.K), s.R);
-    prepare_image_kernel<<<grid, kSlotCodewords, 0, stream>>>(s, cb, sp, mx, p + kPreparedImageOffset);
-    if ((rc = check_launch()) != RVQ_OK) return rc;
-    prepare_finish_kernel<<<1, 32, 0, stream>>>(s, sp, mx);
-    return check_launch();
+    if (rc != RVQ_OK) return rc;
+    if (s.gd == 32) {
+        dim3 grid(slots_per_stage(s.K), s.R);
+        prepare_image_kernel<<<grid, kSlotCodewords, 0, stream>>>(s, cb, sp, mx, p + kPreparedImageOffset);
+        if ((rc = check_launch()) != RVQ_OK) return rc;
+        prepare_finish_kernel<<<1, 32, 0, stream>>>(s, sp, mx);
+        if ((rc = check_launch()) != RVQ_OK) return rc;
+    }
+    if (decode_sliced_supported(s)) {
+        const size_t off = decode_section_offset(s);
+        DecodeParams *dp = reinterpret_cast<DecodeParams *>(p + off);
+        float *lo = reinterpret_cast<float *>(p + off + 128);     // per-stage minima, second half of the parameter block
+        decode_range_kernel<<<8, 256, 0, stream>>>(s, cb, dp, lo);
+        if ((rc = check_launch()) != RVQ_OK) return rc;
+        decode_bias_kernel<<<1, 1, 0, stream>>>(dp, lo);
+        if ((rc = check_launch()) != RVQ_OK) return rc;
+        dim3 grid((s.K + 255) / 256, kDecodeSlices);
+        decode_table_kernel<<<grid, 256, 0, stream>>>(s, cb, dp, lo, reinterpret_cast<uint4 *>(p + off + 256));
+        if ((rc = check_launch()) != RVQ_OK) return rc;
+    }
+    return RVQ_OK;
 }
 
 }  // namespace rvq

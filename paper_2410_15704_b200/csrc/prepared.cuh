@@ -16,7 +16,32 @@ constexpr size_t kPreparedImageOffset = 768;              // operand image, [R][
 
 struct PreparedHeader {
     uint32_t magic, R, K, gd, slots;
+    uint32_t decode_offset;   // byte offset of the decoder section, 0 if absent
 };
+
+// Decoder section (group_dim 32, R <= 8, K <= kDecodeMaxK): per stage an affine
+// map value = lo + (f - 1) * step with f = 1 + q * 2^-15 in [1, 2) the float whose
+// mantissa bits 22..8 are the 15-bit level q, then four channel slices of the
+// codebooks as levels: table[slice][code][stage 0..7][8 channels] uint16, each
+// with bit 15 set (it becomes the lowest exponent bit of f).
+struct DecodeParams {
+    float step[8];    // (max - min) * 32768 / 32767 per stage, 0 for absent stages
+    float bias;       // sum over stages of (min - step)
+    float err;        // bound on |sum of table values - sum of float32 values| per channel
+    float pad[6];
+};
+constexpr int kDecodeMaxK = 1536;                         // 128 bytes per code per slice in shared memory
+constexpr int kDecodeSlices = 4;
+__host__ __device__ inline size_t decode_table_bytes(int K) { return (size_t)kDecodeSlices * K * 128; }
+__host__ __device__ inline bool decode_sliced_supported(const Shape &s)
+{
+    // 16-bit outputs only: their own rounding (2^-9 or 2^-12 relative) dwarfs the table's
+    return s.gd == 32 && s.G == 4 && s.R <= 8 && s.K <= kDecodeMaxK && s.dtype != RVQ_F32;
+}
+__host__ __device__ inline size_t encode_image_bytes(const Shape &s)
+{
+    return s.gd == 32 ? (size_t)s.R * ((s.K + 127) / 128) * 20480 : 0;
+}
 
 struct StageParams {
     float scale;    // 2^k applied to residuals and codewords of this stage

@@ -13,9 +13,10 @@
 //     by its lane, so the 8 lanes of a quarter warp always touch 8 different
 //     16-byte bank groups whatever the codes are.
 //   - A level q becomes the float 1 + q 2^-15 by one byte permute (the stored
-//     level carries the exponent's low bit), and one FMA with the stage's step
-//     adds it to a float32 sum; the affine offsets of all stages are removed at
-//     the end, then the sum is multiplied by the stored deviation and rounded once.
+//     level carries the exponent's low bit), and one packed float32x2 FMA with
+//     the stage's step adds two channels to their float32 sums, which start at
+//     the affine offset of all stages; the sums are then multiplied by the
+//     stored deviation and rounded once.
 //   - With strided groups the 4 lanes of a head vector exchange their results so
 //     that every lane stores 16 contiguous bytes.
 #include "prepared.cuh"
@@ -48,6 +49,17 @@ __device__ __forceinline__ float level_to_float(uint32_t word)
 {
     // bytes of the result, most significant first: 0x3F, half's high byte, half's low byte, 0x00
     return __uint_as_float(__byte_perm(word, 0x3F000000u, H ? 0x7324 : 0x7104));
+}
+
+// Packed float32x2 multiply-add (one instruction for two channels).
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
+{
+    float2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(*reinterpret_cast<unsigned long long *>(&d))
+        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)),
+          "l"(*reinterpret_cast<unsigned long long *>(&c)));
+    return d;
 }
 
 template <int DT>
@@ -103,40 +115,54 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
             }
             cw[0] = a0; cw[1] = a1; cw[2] = a2; cw[3] = a3;
         }
-        float acc[8];
+        // codes out of range (never produced by the encoder): counted, read as code 0
+        {
+            const uint32_t m = __vmaxu2(__vmaxu2(cw[0], cw[1]), __vmaxu2(cw[2], cw[3]));
+            if (max(m & 0xFFFFu, m >> 16) >= (uint32_t)s.K) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t lo = cw[c] & 0xFFFFu, hi = cw[c] >> 16;
+                    if (lo >= (uint32_t)s.K) { lo = 0; ++bad; }
+                    if (hi >= (uint32_t)s.K) { hi = 0; ++bad; }
+                    cw[c] = lo | (hi << 16);
+                }
+            }
+        }
+        // two channels per packed float32x2 accumulator, started at the affine offset
+        float2 acc[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] = make_float2(bias, bias);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
-            if (j >= (uint32_t)s.K) { j = 0; ++bad; }
+            const uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
             const uint4 e = *reinterpret_cast<const uint4 *>(table + j * 128u + unit[k]);
-            const float sk = step[k];
-            acc[0] = fmaf(level_to_float<0>(e.x), sk, acc[0]); acc[1] = fmaf(level_to_float<1>(e.x), sk, acc[1]);
-            acc[2] = fmaf(level_to_float<0>(e.y), sk, acc[2]); acc[3] = fmaf(level_to_float<1>(e.y), sk, acc[3]);
-            acc[4] = fmaf(level_to_float<0>(e.z), sk, acc[4]); acc[5] = fmaf(level_to_float<1>(e.z), sk, acc[5]);
-            acc[6] = fmaf(level_to_float<0>(e.w), sk, acc[6]); acc[7] = fmaf(level_to_float<1>(e.w), sk, acc[7]);
+            const float2 sk = make_float2(step[k], step[k]);
+            acc[0] = fma2(make_float2(level_to_float<0>(e.x), level_to_float<1>(e.x)), sk, acc[0]);
+            acc[1] = fma2(make_float2(level_to_float<0>(e.y), level_to_float<1>(e.y)), sk, acc[1]);
+            acc[2] = fma2(make_float2(level_to_float<0>(e.z), level_to_float<1>(e.z)), sk, acc[2]);
+            acc[3] = fma2(make_float2(level_to_float<0>(e.w), level_to_float<1>(e.w)), sk, acc[3]);
         }
         const float sd = live ? __half2float(__ushort_as_half(std16[v])) : 0.0f;
+        float o8[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = (acc[i] + bias) * sd;
+        for (int i = 0; i < 4; ++i) { o8[2 * i] = acc[i].x * sd; o8[2 * i + 1] = acc[i].y * sd; }
 
         if (DT == RVQ_F32) {
             if (s.layout == RVQ_GROUP_CONTIGUOUS) {
                 if (live) {
                     float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + v * stride + g * 32 + slice * 8);
-                    o[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-                    o[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                    o[0] = make_float4(o8[0], o8[1], o8[2], o8[3]);
+                    o[1] = make_float4(o8[4], o8[5], o8[6], o8[7]);
                 }
             } else if (live) {
                 float *o = reinterpret_cast<float *>(out) + v * stride + slice * 32 + g;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) o[4 * i] = acc[i];         // channel (8 slice + i) * 4 + g
+                for (int i = 0; i < 8; ++i) o[4 * i] = o8[i];         // channel (8 slice + i) * 4 + g
             }
         } else {
             uint32_t w[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) w[c] = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(acc[2 * c], acc[2 * c + 1]);
+            for (int c = 0; c < 4; ++c) w[c] = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(o8[2 * c], o8[2 * c + 1]);
             if (s.layout == RVQ_GROUP_CONTIGUOUS) {
                 if (live)
                     *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(out) + v * stride + g * 32 + slice * 8) =

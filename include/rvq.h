@@ -53,7 +53,8 @@ typedef enum {
     RVQ_ERR_UNSUPPORTED = -3,  /* shape outside what the kernels handle              */
     RVQ_ERR_WORKSPACE = -4,    /* workspace smaller than rvq_workspace_bytes()       */
     RVQ_ERR_LAUNCH = -5,       /* the CUDA runtime refused a launch or a copy        */
-    RVQ_ERR_DEVICE = -6        /* not an sm_100 device, or no device                 */
+    RVQ_ERR_DEVICE = -6,       /* not an sm_100 device, or no device                 */
+    RVQ_ERR_STATIC_LIMIT = -7  /* shape needs more than the library's built-in scratch */
 } rvq_error;
 
 /* Shape of one quantizer (Section 3: default dim 128, group_dim 32, depth 8,
@@ -205,6 +206,41 @@ int rvq_ema_stats(const rvq_config *cfg /* host */, const void *x, int64_t n, in
 int rvq_ema_apply(const rvq_config *cfg /* host */, const float *batch_count,
                   const float *batch_sum, float *codebooks, float *ema_count, float *ema_sum,
                   float decay, float eps, void *stream /* cudaStream_t */);
+
+/*
+ * rvq_ema_update without a workspace argument.  (The paper has no counterpart;
+ * this exists for one kind of caller.)
+ *
+ * Who it is for: code that may not, or cannot, get device memory at the moment
+ * it needs the update -- a plugin running inside a host application that owns
+ * the allocator and hands out only the input and output buffers, a step inside
+ * a region where cudaMalloc is forbidden because it synchronises the device, or
+ * a process whose memory budget was fixed at start-up.  rvq_ema_update asks such
+ * a caller for rvq_workspace_bytes() of scratch it has no way to provide.
+ *
+ * Here the scratch is a fixed array inside the library
+ * (rvq_ema_static_scratch_bytes(), about 2.1 MiB; every GPU that loads the
+ * library holds it until the process ends).  Shapes whose rvq_workspace_bytes()
+ * is larger -- more than depth 8 x 2048 codes x 32 channels' worth -- are
+ * refused with RVQ_ERR_STATIC_LIMIT and nothing is launched.  The call itself
+ * allocates and frees nothing.
+ *
+ * Arguments, results and error codes are those of rvq_ema_update.  Differences:
+ *   - The first call on each device looks up the array's device address (a
+ *     runtime query, not a launch).  Make that first call outside any stream
+ *     capture.
+ *   - All calls, on every stream, share the one array, and it still holds the
+ *     previous call's numbers when the next begins; each call clears the parts
+ *     it accumulates into.  Two calls that can overlap on the GPU (different
+ *     streams without an ordering between them) corrupt each other: order them.
+ */
+int rvq_ema_update_static(const rvq_config *cfg /* host */, const void *x, int64_t n,
+                          int64_t x_row_stride, const void *codes, float *codebooks,
+                          float *ema_count, float *ema_sum, float *batch_count, float decay,
+                          float eps, rvq_status *status, void *stream /* cudaStream_t */);
+
+/* Size in bytes of the scratch array behind rvq_ema_update_static. */
+size_t rvq_ema_static_scratch_bytes(void);
 
 #ifdef __cplusplus
 }

@@ -68,12 +68,16 @@ def _load() -> ctypes.CDLL:
     lib.rvq_ema_stats.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.rvq_ema_apply.restype = ctypes.c_int
     lib.rvq_ema_apply.argtypes = [cfgp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp]
+    lib.rvq_ema_update_static.restype = ctypes.c_int
+    lib.rvq_ema_update_static.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, ctypes.c_float,
+                                          ctypes.c_float, vp, vp]
+    lib.rvq_ema_static_scratch_bytes.restype = sz
     return lib
 
 
 lib = _load()
 
-EXPORTS = ("rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
+EXPORTS = ("rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
            "rvq_prepare_codebooks", "rvq_workspace_bytes", "rvq_encode", "rvq_decode",
            "rvq_ema_update")
 
@@ -184,6 +188,23 @@ def rvq_ema_apply(cfg, batch_count, batch_sum, codebooks, ema_count, ema_sum, de
     if check:
         _check(rc, "rvq_ema_apply")
     return rc
+
+
+def rvq_ema_update_static(cfg, x, n, x_row_stride, codes, codebooks, ema_count, ema_sum, batch_count,
+                          decay, eps, status=None, stream=None, check=True) -> int:
+    """rvq_ema_update with the library's own fixed scratch: no workspace to pass, nothing
+    allocated.  For callers that cannot obtain device memory themselves; see include/rvq.h
+    for the size limit and for why overlapping calls must be ordered."""
+    rc = lib.rvq_ema_update_static(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codes), _ptr(codebooks),
+                                   _ptr(ema_count), _ptr(ema_sum), _ptr(batch_count), decay, eps,
+                                   _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_ema_update_static")
+    return rc
+
+
+def rvq_ema_static_scratch_bytes() -> int:
+    return int(lib.rvq_ema_static_scratch_bytes())
 
 
 def rvq_launch_count() -> int:

@@ -62,6 +62,7 @@ const char *rvq_status_string(int code)
     case RVQ_ERR_WORKSPACE: return "workspace too small";
     case RVQ_ERR_LAUNCH: return "CUDA launch failed";
     case RVQ_ERR_DEVICE: return "no sm_100 device";
+    case RVQ_ERR_STATIC_LIMIT: return "shape needs more scratch than the library's built-in array holds";
     default: return "unknown error";
     }
 }

@@ -147,3 +147,74 @@ int launch_ema_apply(const Shape &s, const float *batch_count, const float *batc
 }
 
 }  // namespace rvq
+
+// ---------------------------------------------------------------------------
+// rvq_ema_update_static: the same update with its scratch inside the library.
+//
+// The scratch of rvq_ema_update (integer counts, batch counts, batch sums) lives
+// here in a fixed device array instead of a caller buffer, so a caller that has
+// no way to obtain device memory of its own can still run the update.  The array
+// is part of the library image: every GPU that loads the library carries it until
+// the process exits, used or not.
+namespace {
+
+// Room for depth 8 x 2048 codes x 32 channels (the paper's default quantizer):
+// 64 KiB of counts + 64 KiB of batch counts + 2 MiB of batch sums.
+constexpr size_t kStaticScratchBytes = 65536 + 65536 + 2097152;
+static __device__ __align__(256) unsigned char g_ema_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void *g_scratch_addr[kMaxDevices];      // device address of g_ema_scratch per device ordinal (null: not looked up yet)
+
+// The array's name is only a handle on the host; the address a kernel can use
+// has to be asked for, once per device, with that device current.
+int static_scratch(void **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RVQ_ERR_DEVICE;
+    if (!g_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_ema_scratch) != cudaSuccess || !ptr) return RVQ_ERR_DEVICE;
+        g_scratch_addr[dev] = ptr;
+    }
+    *out = g_scratch_addr[dev];
+    return RVQ_OK;
+}
+
+}  // namespace
+
+extern "C" size_t rvq_ema_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+extern "C" int rvq_ema_update_static(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                                     const void *codes, float *codebooks, float *ema_count, float *ema_sum,
+                                     float *batch_count, float decay, float eps, rvq_status *status,
+                                     void *stream)
+{
+    using namespace rvq;
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if (n < 0 || x_row_stride < s.dim || (n > 0 && (!x || !codes))) return RVQ_ERR_BADARG;
+    if (!codebooks || !ema_count || !ema_sum) return RVQ_ERR_BADARG;
+    if (!(decay >= 0.0f && decay <= 1.0f) || !(eps >= 0.0f)) return RVQ_ERR_BADARG;
+    if (!aligned16(x) || (x_row_stride * s.elem_bytes) % 16 || !aligned16(codes) || !aligned16(codebooks) ||
+        !aligned16(ema_sum))
+        return RVQ_ERR_ALIGN;
+    if (ema_workspace_bytes(s) > kStaticScratchBytes) return RVQ_ERR_STATIC_LIMIT;
+    void *scratch = nullptr;
+    if ((rc = static_scratch(&scratch)) != RVQ_OK) return rc;
+    // same carving as rvq_ema_update: counts | batch counts | batch sums
+    uint8_t *ws = reinterpret_cast<uint8_t *>(scratch);
+    float *bc = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s));
+    float *bs = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s) + round256((size_t)s.R * s.K * sizeof(float)));
+    // launch_ema_stats zeroes the counts and the batch sums it accumulates into;
+    // nothing else in the scratch is read before it is written
+    rc = launch_ema_stats(s, x, n, x_row_stride, codes, codebooks, bc, bs, scratch, status, (cudaStream_t)stream);
+    if (rc != RVQ_OK) return rc;
+    if (batch_count &&
+        cudaMemcpyAsync(batch_count, bc, (size_t)s.R * s.K * sizeof(float), cudaMemcpyDeviceToDevice,
+                        (cudaStream_t)stream) != cudaSuccess)
+        return RVQ_ERR_LAUNCH;
+    return launch_ema_apply(s, bc, bs, codebooks, ema_count, ema_sum, decay, eps, (cudaStream_t)stream);
+}
+

@@ -69,22 +69,25 @@ counts_to_float_kernel(const uint32_t *__restrict__ cnt, float *__restrict__ out
     if (t < total) out[t] = (float)cnt[t];
 }
 
-// One block per stage: N <- decay N + (1-decay) n, total = sum_j N, then
-// M <- decay M + (1-decay) m and C = M / ((N + eps) total / (total + K eps)).
+// N <- decay N + (1-decay) n, element-wise.
 __global__ void __launch_bounds__(256)
-ema_apply_kernel(Shape s, const float *__restrict__ cnt, const float *__restrict__ sum,
-                 float *__restrict__ cb, float *__restrict__ ema_count,
-                 float *__restrict__ ema_sum, float decay, float eps)
+ema_count_kernel(const float *__restrict__ cnt, float *__restrict__ ema_count, int total, float decay)
+{
+    const int t = blockIdx.x * 256 + threadIdx.x;
+    if (t < total) ema_count[t] = decay * ema_count[t] + (1.0f - decay) * cnt[t];
+}
+
+// grid (parts, R): every block sums the stage's updated counts (same order in
+// every block, so all blocks of a stage get the same total), then updates its
+// share of M <- decay M + (1-decay) m and C = M / ((N + eps) total / (total + K eps)).
+__global__ void __launch_bounds__(256)
+ema_apply_kernel(Shape s, const float *__restrict__ sum, float *__restrict__ cb,
+                 const float *__restrict__ ema_count, float *__restrict__ ema_sum, float decay, float eps)
 {
     __shared__ float red[256];
-    const int r = blockIdx.x, tid = threadIdx.x;
+    const int r = blockIdx.y, tid = threadIdx.x;
     float local = 0.0f;
-    for (int j = tid; j < s.K; j += 256) {
-        const size_t p = (size_t)r * s.K + j;
-        const float nn = decay * ema_count[p] + (1.0f - decay) * cnt[p];
-        ema_count[p] = nn;
-        local += nn;
-    }
+    for (int j = tid; j < s.K; j += 256) local += ema_count[(size_t)r * s.K + j];
     red[tid] = local;
     __syncthreads();
     for (int w = 128; w > 0; w >>= 1) {
@@ -93,8 +96,9 @@ ema_apply_kernel(Shape s, const float *__restrict__ cnt, const float *__restrict
     }
     const float tot = red[0];
     const float scale = tot / (tot + (float)s.K * eps);
-    for (int t = tid; t < s.K * s.gd; t += 256) {
-        const size_t p = (size_t)r * s.K * s.gd + t;
+    const int per_stage = s.K * s.gd;
+    for (int t = blockIdx.x * 256 + tid; t < per_stage; t += gridDim.x * 256) {
+        const size_t p = (size_t)r * per_stage + t;
         const int j = t / s.gd;
         const float mm = decay * ema_sum[p] + (1.0f - decay) * sum[p];
         ema_sum[p] = mm;
@@ -142,7 +146,13 @@ int launch_ema_stats(const Shape &s, const void *x, int64_t n, int64_t stride, c
 int launch_ema_apply(const Shape &s, const float *batch_count, const float *batch_sum, float *cb,
                      float *ema_count, float *ema_sum, float decay, float eps, cudaStream_t stream)
 {
-    ema_apply_kernel<<<s.R, 256, 0, stream>>>(s, batch_count, batch_sum, cb, ema_count, ema_sum, decay, eps);
+    const int bins = s.R * s.K;
+    ema_count_kernel<<<(bins + 255) / 256, 256, 0, stream>>>(batch_count, ema_count, bins, decay);
+    int rc = check_launch();
+    if (rc != RVQ_OK) return rc;
+    int parts = (s.K * s.gd + 256 * 8 - 1) / (256 * 8);
+    if (parts > 32) parts = 32;
+    ema_apply_kernel<<<dim3(parts, s.R), 256, 0, stream>>>(s, batch_sum, cb, ema_count, ema_sum, decay, eps);
     return check_launch();
 }
 

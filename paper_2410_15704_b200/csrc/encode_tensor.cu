@@ -419,6 +419,22 @@ encode_tensor_kernel(const Params p)
 
 #pragma unroll 1
                 for (int c = 0; c < S && ok; ++c) {
+                    if (c == S - 1 && w.cnt > 0) {
+                        // Before the last chunk the running winner is the final one most of the time:
+                        // start fetching its cell's three codewords while the MMA chain runs.
+                        int pb = 0, pq = 0;
+#pragma unroll
+                        for (int e = kListCap - 1; e >= 0; --e)
+                            if (e < w.cnt && list_v[e * kRowsPerPass] == w.m1) pb = list_i[e * kRowsPerPass];
+#pragma unroll
+                        for (int q = 10; q >= 0; --q)
+                            if (w.d[q] == w.m1) pq = q;
+                        const int pj = min(pb * 32 + 3 * pq, s.K - 1);
+                        const float *pp = cbr + (size_t)pj * 32;
+                        asm volatile("prefetch.global.L1 [%0];" ::"l"(pp));
+                        asm volatile("prefetch.global.L1 [%0];" ::"l"(pp + 32));
+                        asm volatile("prefetch.global.L1 [%0];" ::"l"(pp + 64));
+                    }
                     ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag);
                     ok = __all_sync(0xFFFFFFFFu, ok);          // tcgen05.ld below needs the whole warp
                     ++chunk_use;
@@ -514,6 +530,21 @@ encode_tensor_kernel(const Params p)
                 // every listed block of one such row at a time (or all columns when the list
                 // overflowed), then reduces to the smallest distance, lowest index on ties.
                 uint32_t todo = __ballot_sync(0xFFFFFFFFu, flagged);
+                // first touch every codeword the loop below will read, so that their loads overlap
+                for (uint32_t pre = todo; pre; pre &= pre - 1) {
+                    const int src = __ffs(pre) - 1;
+                    const float lim_s = __shfl_sync(0xFFFFFFFFu, lim, src);
+                    const int cnt_s = __shfl_sync(0xFFFFFFFFu, cnt, src);
+                    const bool all_s = __shfl_sync(0xFFFFFFFFu, (int)scan_all, src) != 0;
+                    const int row_s = rloc - lane + src;
+                    if (all_s) continue;
+                    for (int e = 0; e < cnt_s; ++e) {
+                        const float fv = reinterpret_cast<const float *>(smem + kOffListV)[e * kRowsPerPass + row_s];
+                        if (!(fv <= lim_s)) continue;
+                        const int j = (int)reinterpret_cast<const uint16_t *>(smem + kOffListI)[e * kRowsPerPass + row_s] * 32 + lane;
+                        if (j < s.K) asm volatile("prefetch.global.L1 [%0];" ::"l"(cbr + (size_t)j * 32));
+                    }
+                }
                 while (todo) {
                     const int src = __ffs(todo) - 1;
                     todo &= todo - 1;

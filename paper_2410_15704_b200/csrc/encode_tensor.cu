@@ -206,15 +206,25 @@ __device__ __forceinline__ void list_block(Sweep &w, float cb_min, int block, fl
     w.cnt += app ? 1 : 0;
 }
 
+// 32-byte read-only global load: a codeword row costs four of these, and for
+// row-per-lane gathers it is the number of load instructions that the L1 pays for.
+__device__ __forceinline__ void ldg256(const float *p, float (&v)[8])
+{
+    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p));
+}
+
 // Exact squared distance, direct form, same operation order as the scalar kernel.
 __device__ __forceinline__ float exact_distance(const float (&z)[32], const float *__restrict__ e)
 {
     float acc = 0.0f;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        const float4 ev = __ldg(reinterpret_cast<const float4 *>(e) + q);
-        const float t0 = z[4 * q] - ev.x, t1 = z[4 * q + 1] - ev.y, t2 = z[4 * q + 2] - ev.z, t3 = z[4 * q + 3] - ev.w;
-        acc = fmaf(t0, t0, acc); acc = fmaf(t1, t1, acc); acc = fmaf(t2, t2, acc); acc = fmaf(t3, t3, acc);
+    for (int q = 0; q < 4; ++q) {
+        float ev[8];
+        ldg256(e + 8 * q, ev);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { const float t = z[8 * q + k] - ev[k]; acc = fmaf(t, t, acc); }
     }
     return acc;
 }
@@ -506,19 +516,20 @@ encode_tensor_kernel(const Params p)
                     // the three columns of the cell, scored together so that their loads overlap
                     const int j0 = b1 * 32 + 3 * q1;
                     const bool in1 = 3 * q1 + 1 < 32 && j0 + 1 < s.K, in2 = 3 * q1 + 2 < 32 && j0 + 2 < s.K;
-                    const float4 *e0 = reinterpret_cast<const float4 *>(cbr + (size_t)(j0 < s.K ? j0 : 0) * 32);
-                    const float4 *e1 = in1 ? e0 + 8 : e0, *e2 = in2 ? e0 + 16 : e0;
+                    const float *e0 = cbr + (size_t)(j0 < s.K ? j0 : 0) * 32;
+                    const float *e1 = in1 ? e0 + 32 : e0, *e2 = in2 ? e0 + 64 : e0;
                     float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f;
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 u0 = __ldg(e0 + q), u1 = __ldg(e1 + q), u2 = __ldg(e2 + q);
-                        float t;
-                        t = z[4 * q] - u0.x; a0 = fmaf(t, t, a0); t = z[4 * q + 1] - u0.y; a0 = fmaf(t, t, a0);
-                        t = z[4 * q + 2] - u0.z; a0 = fmaf(t, t, a0); t = z[4 * q + 3] - u0.w; a0 = fmaf(t, t, a0);
-                        t = z[4 * q] - u1.x; a1 = fmaf(t, t, a1); t = z[4 * q + 1] - u1.y; a1 = fmaf(t, t, a1);
-                        t = z[4 * q + 2] - u1.z; a1 = fmaf(t, t, a1); t = z[4 * q + 3] - u1.w; a1 = fmaf(t, t, a1);
-                        t = z[4 * q] - u2.x; a2 = fmaf(t, t, a2); t = z[4 * q + 1] - u2.y; a2 = fmaf(t, t, a2);
-                        t = z[4 * q + 2] - u2.z; a2 = fmaf(t, t, a2); t = z[4 * q + 3] - u2.w; a2 = fmaf(t, t, a2);
+                    for (int q = 0; q < 4; ++q) {
+                        float u0[8], u1[8], u2[8];
+                        ldg256(e0 + 8 * q, u0); ldg256(e1 + 8 * q, u1); ldg256(e2 + 8 * q, u2);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            float t;
+                            t = z[8 * q + k] - u0[k]; a0 = fmaf(t, t, a0);
+                            t = z[8 * q + k] - u1[k]; a1 = fmaf(t, t, a1);
+                            t = z[8 * q + k] - u2[k]; a2 = fmaf(t, t, a2);
+                        }
                     }
                     if (j0 < s.K) { best = a0; bj = j0; }
                     if (in1 && a1 < best) { best = a1; bj = j0 + 1; }
@@ -584,11 +595,13 @@ encode_tensor_kernel(const Params p)
                 }
                 if (deg) bj = 0;
                 if (!deg) {
-                    const float4 *e4 = reinterpret_cast<const float4 *>(cbr + (size_t)bj * 32);
+                    const float *ew = cbr + (size_t)bj * 32;
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 ev = __ldg(e4 + q);
-                        z[4 * q] -= ev.x; z[4 * q + 1] -= ev.y; z[4 * q + 2] -= ev.z; z[4 * q + 3] -= ev.w;
+                    for (int q = 0; q < 4; ++q) {
+                        float ev[8];
+                        ldg256(ew + 8 * q, ev);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) z[8 * q + k] -= ev[k];
                     }
                 }
                 codes_s[rloc * 16 + r] = (uint16_t)bj;

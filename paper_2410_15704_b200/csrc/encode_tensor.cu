@@ -1,7 +1,8 @@
 // Tensor-core encode for group_dim 32 (Section 2.2, Algorithm 1).
 //
-// One persistent CTA per SM works on passes of 384 group rows (three tiles of 128
-// rows, one row per thread, 12 epilogue warps) plus four single-thread roles in
+// One persistent CTA per SM takes a contiguous run of 128-row tiles and works
+// through it in rounds of up to three tiles (one row per thread, 12 epilogue
+// warps; rounds are sized evenly, e.g. 7 tiles = 3 + 2 + 2) plus four single-thread roles in
 // warps of their own: one MMA issuer per tile and the operand loader.
 //   - Scores ||e||^2 - 2 z.e of a 128-row tile against 128 codewords are one
 //     tcgen05.mma chain (M=128, N=128, seven K=16 steps over the split
@@ -238,7 +239,14 @@ struct Params {
     void *codes;
     uint16_t *std16;
     rvq_status *st;
-    int passes;
+    int tiles;          // 128-row tiles in the whole problem
+};
+
+// The tiles of one CTA: a contiguous run, done in `rounds` rounds of nearly equal size (<= kTiles).
+struct Work {
+    int first, count, rounds;
+    __device__ __forceinline__ int round_size(int k) const { return count / rounds + (k < count % rounds ? 1 : 0); }
+    __device__ __forceinline__ int round_first(int k) const { return first + k * (count / rounds) + min(k, count % rounds); }
 };
 
 // 17 warps are granted registers as 20 (whole groups of four): 96 per thread.
@@ -253,7 +261,14 @@ encode_tensor_kernel(const Params p)
     const Shape &s = p.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = slots_per_stage(s.K);
-    const int my_passes = (p.passes - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    Work work;
+    {
+        const int per = p.tiles / (int)gridDim.x, rem = p.tiles % (int)gridDim.x, b = (int)blockIdx.x;
+        work.count = per + (b < rem ? 1 : 0);
+        work.first = b * per + min(b, rem);
+        work.rounds = (work.count + kTiles - 1) / kTiles;
+    }
+    const int my_passes = work.rounds;
     const StageParams *sp = reinterpret_cast<const StageParams *>(p.prepared + kPreparedParamsOffset);
     const uint8_t *image = p.prepared + kPreparedImageOffset;
     const uint32_t bar0 = smem_u32(bars);
@@ -319,13 +334,23 @@ encode_tensor_kernel(const Params p)
             const uint64_t ones_desc = make_smem_desc(smem_u32(smem + kOffA), 2048, 128);
             const uint32_t acc = tmem + t * kTileCols, a0 = acc + 128;
             const uint32_t bar_ready = BAR(kBarAReady + t), bar_free = BAR(kBarAccFree + t), bar_acc = BAR(kBarAccFull + t);
-            uint32_t slot = 0, full_par = 0, s_in = 0, ready_par = 0, free_par = 1;
-            bool ok = true;
+            const uint32_t per_round = (uint32_t)s.R * (uint32_t)S;
+            uint32_t slot = 0, full_par = 0, s_in = 0, ready_par = 0, free_par = 1, in_round = 0;
+            int round = 0;
+            bool ok = true, first = true, active = t < work.round_size(0);
             for (uint32_t q = 0; q < total && ok; ++q) {
                 ok = mbar_wait(BAR(kBarFull + slot), full_par, abort_flag);
+                if (!active) {
+                    // this tile sits the round out, but the slot still waits for its release
+                    if (ok) mbar_arrive(BAR(kBarEmpty + slot));
+                    if (++slot == (uint32_t)kRing) { slot = 0; full_par ^= 1u; }
+                    if (++in_round == per_round) { in_round = 0; ++round; active = round < work.rounds && t < work.round_size(round); }
+                    continue;
+                }
                 if (ok && s_in == 0) ok = mbar_wait(bar_ready, ready_par, abort_flag);
-                if (ok && q > 0) ok = mbar_wait(bar_free, free_par, abort_flag);
+                if (ok && !first) ok = mbar_wait(bar_free, free_par, abort_flag);
                 if (!ok) break;
+                first = false;
                 tc_fence_after();
                 const uint64_t bd = bdesc0 + (uint64_t)(slot * (uint32_t)(kSlotBytes >> 4));
                 mma_f16_ts(acc, a0, bd, idesc, 0);                      // hi[0:16]  . hi cells 0-1
@@ -340,6 +365,7 @@ encode_tensor_kernel(const Params p)
                 free_par ^= 1u;
                 if (++slot == (uint32_t)kRing) { slot = 0; full_par ^= 1u; }
                 if (++s_in == (uint32_t)S) { s_in = 0; ready_par ^= 1u; }
+                if (++in_round == per_round) { in_round = 0; ++round; active = round < work.rounds && t < work.round_size(round); }
             }
         }
     } else {
@@ -357,8 +383,9 @@ encode_tensor_kernel(const Params p)
         bool ok = true;
 
         for (int pass = 0; pass < my_passes && ok; ++pass) {
-            const int64_t row0 = ((int64_t)blockIdx.x + (int64_t)pass * gridDim.x) * kRowsPerPass;
-            const int64_t grow = row0 + rloc;
+            if (tile >= work.round_size(pass)) continue;            // this tile sits the round out
+            const int64_t row0 = (int64_t)(work.round_first(pass) + tile) * 128;   // first row of this tile
+            const int64_t grow = row0 + q4 * 32 + lane;
             const int64_t v = grow / G;
             const int g = (int)(grow - v * G);
             const bool valid = v < p.n;
@@ -625,7 +652,7 @@ encode_tensor_kernel(const Params p)
                 const int wrow0 = rloc - lane;
                 for (int t = lane; t < vec_per_warp * words; t += 32) {
                     const int vl = t / words, w = t - vl * words;
-                    const int64_t vv = (row0 + wrow0) / G + vl;
+                    const int64_t vv = (row0 + q4 * 32) / G + vl;
                     if (vv >= p.n) continue;
                     uint32_t word = 0;
                     const int k_lo = (32 * w) / s.bits, k_hi = min(s.per_vector - 1, (32 * w + 31) / s.bits);
@@ -670,16 +697,17 @@ int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t strid
 {
     if (n == 0) return RVQ_OK;
     const int64_t rows = n * s.G;
-    const int64_t passes = (rows + kRowsPerPass - 1) / kRowsPerPass;
-    if (passes > 0x7FFFFFFF) return RVQ_ERR_UNSUPPORTED;
+    const int64_t tiles = (rows + 127) / 128;
+    if (tiles > 0x7FFFFFFF) return RVQ_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return RVQ_ERR_DEVICE;
     if (cudaFuncSetAttribute(encode_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
-    Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)passes};
-    const int grid = (int)(passes < sms ? passes : sms);
+    Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)tiles};
+    const int64_t groups = (tiles + kTiles - 1) / kTiles;
+    const int grid = (int)(groups < sms ? groups : sms);
     encode_tensor_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);
     return check_launch();
 }

@@ -36,41 +36,6 @@ size_t prepared_bytes(const Shape &s)
     return (b + 255) / 256 * 256;
 }
 
-// One block per stage (8 blocks): range of the stage's entries -> affine map.
-__global__ void __launch_bounds__(256)
-decode_range_kernel(Shape s, const float *__restrict__ cb, DecodeParams *dp, float *lo_out)
-{
-    __shared__ float smin[256], smax[256];
-    const int r = blockIdx.x, tid = threadIdx.x;
-    float lo = INFINITY, hi = -INFINITY;
-    if (r < s.R)
-        for (int t = tid; t < s.K * 32; t += 256) {
-            const float v = cb[(size_t)r * s.K * 32 + t];
-            lo = fminf(lo, v); hi = fmaxf(hi, v);
-        }
-    smin[tid] = lo; smax[tid] = hi;
-    __syncthreads();
-    for (int w = 128; w > 0; w >>= 1) {
-        if (tid < w) { smin[tid] = fminf(smin[tid], smin[tid + w]); smax[tid] = fmaxf(smax[tid], smax[tid + w]); }
-        __syncthreads();
-    }
-    if (tid == 0) {
-        float step = 0.0f, l = 0.0f;
-        if (r < s.R && smax[0] > smin[0]) { l = smin[0]; step = (smax[0] - smin[0]) * (32768.0f / 32767.0f); }
-        else if (r < s.R) { l = smin[0]; }
-        dp->step[r] = step;
-        lo_out[r] = l;
-    }
-}
-
-__global__ void decode_bias_kernel(DecodeParams *dp, const float *lo)
-{
-    float b = 0.0f, e = 0.0f;
-    for (int r = 0; r < 8; ++r) { b += lo[r] - dp->step[r]; e += dp->step[r] * 1.52587890625e-5f; }   // half a level per stage
-    dp->bias = b;
-    dp->err = e;
-}
-
 // One thread per (slice, code): 8 stages x 8 channels of levels.
 __global__ void __launch_bounds__(256)
 decode_table_kernel(Shape s, const float *__restrict__ cb, const DecodeParams *__restrict__ dp,
@@ -98,28 +63,59 @@ decode_table_kernel(Shape s, const float *__restrict__ cb, const DecodeParams *_
 }
 
 
-// One block per stage: largest squared norm -> scale exponent; clears the maxima.
+// grid (kPrepareParts, R): largest squared norm and entry range of a share of one stage's codewords.
 __global__ void __launch_bounds__(256)
-prepare_scale_kernel(Shape s, const float *__restrict__ cb, PreparedHeader *hdr, StageParams *sp,
-                     StageMaxima *mx)
+prepare_reduce_kernel(Shape s, const float *__restrict__ cb, StagePartial *part)
 {
-    __shared__ double red[256];
-    const int r = blockIdx.x, tid = threadIdx.x;
+    __shared__ double rn[256];
+    __shared__ float rlo[256], rhi[256];
+    const int r = blockIdx.y, tid = threadIdx.x;
+    const int per = (s.K + kPrepareParts - 1) / kPrepareParts;
+    const int j0 = blockIdx.x * per, j1 = min(s.K, j0 + per);
     double m = 0.0;
-    for (int j = tid; j < s.K; j += 256) {
+    float lo = INFINITY, hi = -INFINITY;
+    for (int j = j0 + tid; j < j1; j += 256) {
         const float *e = cb + ((size_t)r * s.K + j) * s.gd;
         double acc = 0.0;
-        for (int i = 0; i < s.gd; ++i) acc += (double)e[i] * (double)e[i];
+        for (int i = 0; i < s.gd; ++i) {
+            const float v = e[i];
+            acc += (double)v * (double)v;
+            lo = fminf(lo, v); hi = fmaxf(hi, v);
+        }
         m = fmax(m, acc);
     }
-    red[tid] = m;
+    rn[tid] = m; rlo[tid] = lo; rhi[tid] = hi;
     __syncthreads();
     for (int w = 128; w > 0; w >>= 1) {
-        if (tid < w) red[tid] = fmax(red[tid], red[tid + w]);
+        if (tid < w) {
+            rn[tid] = fmax(rn[tid], rn[tid + w]);
+            rlo[tid] = fminf(rlo[tid], rlo[tid + w]); rhi[tid] = fmaxf(rhi[tid], rhi[tid + w]);
+        }
         __syncthreads();
     }
     if (tid == 0) {
-        const double maxn = red[0];
+        StagePartial &o = part[r * kPrepareParts + blockIdx.x];
+        o.max_norm2 = rn[0]; o.lo = rlo[0]; o.hi = rhi[0];
+    }
+}
+
+// One block, thread r per stage: scale exponent from the largest squared norm, the decoder's
+// affine map from the entry range; clears the maxima the image kernel accumulates into.
+__global__ void __launch_bounds__(32)
+prepare_params_kernel(Shape s, const StagePartial *__restrict__ part, PreparedHeader *hdr, StageParams *sp,
+                      StageMaxima *mx, DecodeParams *dp, float *dec_lo)
+{
+    __shared__ float s_lo[8], s_step[8];
+    const int r = threadIdx.x;
+    if (r < 8) { s_lo[r] = 0.0f; s_step[r] = 0.0f; }
+    __syncwarp();
+    if (r < s.R) {
+        double maxn = 0.0;
+        float lo = INFINITY, hi = -INFINITY;
+        for (int q = 0; q < kPrepareParts; ++q) {
+            const StagePartial &pp = part[r * kPrepareParts + q];
+            maxn = fmax(maxn, pp.max_norm2); lo = fminf(lo, pp.lo); hi = fmaxf(hi, pp.hi);
+        }
         int k = 12;
         if (maxn > 0.0 && isfinite(maxn)) {
             k = (int)floor(0.5 * log2(8192.0 / maxn));
@@ -130,11 +126,21 @@ prepare_scale_kernel(Shape s, const float *__restrict__ cb, PreparedHeader *hdr,
         sp[r].b = INFINITY;
         sp[r].unsafe = (!isfinite(maxn) || ldexp(maxn, 2 * k) > 8200.0) ? 1.0f : 0.0f;
         mx[r].emax = 0u; mx[r].eerr = 0u; mx[r].nmax = 0u; mx[r].elomax = 0u;
-        if (r == 0) {
-            hdr->magic = kPreparedMagic; hdr->R = s.R; hdr->K = s.K; hdr->gd = s.gd;
-            hdr->slots = slots_per_stage(s.K);
-            hdr->decode_offset = decode_sliced_supported(s)
-                ? (uint32_t)((kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256) : 0u;
+        if (r < 8) { s_lo[r] = lo; s_step[r] = hi > lo ? (hi - lo) * (32768.0f / 32767.0f) : 0.0f; }
+    }
+    __syncwarp();
+    if (r == 0) {
+        hdr->magic = kPreparedMagic; hdr->R = s.R; hdr->K = s.K; hdr->gd = s.gd;
+        hdr->slots = slots_per_stage(s.K);
+        hdr->decode_offset = decode_sliced_supported(s)
+            ? (uint32_t)((kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256) : 0u;
+        if (dp) {
+            float b = 0.0f, e = 0.0f;
+            for (int q = 0; q < 8; ++q) {
+                dp->step[q] = s_step[q]; dec_lo[q] = s_lo[q];
+                b += s_lo[q] - s_step[q]; e += s_step[q] * 1.52587890625e-5f;       // half a level per stage
+            }
+            dp->bias = b; dp->err = e;
         }
     }
 }
@@ -216,9 +222,16 @@ int launch_prepare(const Shape &s, const float *cb, void *prepared, cudaStream_t
     PreparedHeader *hdr = reinterpret_cast<PreparedHeader *>(p);
     StageParams *sp = reinterpret_cast<StageParams *>(p + kPreparedParamsOffset);
     StageMaxima *mx = reinterpret_cast<StageMaxima *>(p + kPreparedMaximaOffset);
-    prepare_scale_kernel<<<s.R, 256, 0, stream>>>(s, cb, hdr, sp, mx);
+    StagePartial *part = reinterpret_cast<StagePartial *>(p + kPreparedPartialsOffset);
+    const bool dec = decode_sliced_supported(s);
+    const size_t off = decode_section_offset(s);
+    DecodeParams *dp = dec ? reinterpret_cast<DecodeParams *>(p + off) : nullptr;
+    float *lo = dec ? reinterpret_cast<float *>(p + off + 128) : nullptr;   // per-stage minima, second half of the parameter block
+    prepare_reduce_kernel<<<dim3(kPrepareParts, s.R), 256, 0, stream>>>(s, cb, part);
     int rc = check_launch();
     if (rc != RVQ_OK) return rc;
+    prepare_params_kernel<<<1, 32, 0, stream>>>(s, part, hdr, sp, mx, dp, lo);
+    if ((rc = check_launch()) != RVQ_OK) return rc;
     if (s.gd == 32) {
         dim3 grid(slots_per_stage(s.K), s.R);
         prepare_image_kernel<<<grid, kSlotCodewords, 0, stream>>>(s, cb, sp, mx, p + kPreparedImageOffset);
@@ -226,14 +239,7 @@ int launch_prepare(const Shape &s, const float *cb, void *prepared, cudaStream_t
         prepare_finish_kernel<<<1, 32, 0, stream>>>(s, sp, mx);
         if ((rc = check_launch()) != RVQ_OK) return rc;
     }
-    if (decode_sliced_supported(s)) {
-        const size_t off = decode_section_offset(s);
-        DecodeParams *dp = reinterpret_cast<DecodeParams *>(p + off);
-        float *lo = reinterpret_cast<float *>(p + off + 128);     // per-stage minima, second half of the parameter block
-        decode_range_kernel<<<8, 256, 0, stream>>>(s, cb, dp, lo);
-        if ((rc = check_launch()) != RVQ_OK) return rc;
-        decode_bias_kernel<<<1, 1, 0, stream>>>(dp, lo);
-        if ((rc = check_launch()) != RVQ_OK) return rc;
+    if (dec) {
         dim3 grid((s.K + 255) / 256, kDecodeSlices);
         decode_table_kernel<<<grid, 256, 0, stream>>>(s, cb, dp, lo, reinterpret_cast<uint4 *>(p + off + 256));
         if ((rc = check_launch()) != RVQ_OK) return rc;

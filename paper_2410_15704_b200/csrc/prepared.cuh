@@ -12,7 +12,9 @@ constexpr int kSlotCells = 10;                            // hi (4), lo (4), nor
 constexpr int kSlotBytes = kSlotCells * kSlotCodewords * 16;   // 20480
 constexpr size_t kPreparedParamsOffset = 256;             // StageParams[16]
 constexpr size_t kPreparedMaximaOffset = 512;             // StageMaxima[16]
-constexpr size_t kPreparedImageOffset = 768;              // operand image, [R][slots][kSlotBytes]
+constexpr size_t kPreparedPartialsOffset = 768;           // StagePartial[16 stages][kPrepareParts], scratch of the prepare step
+constexpr int kPrepareParts = 16;
+constexpr size_t kPreparedImageOffset = 768 + 16 * 16 * 16;   // operand image, [R][slots][kSlotBytes]
 
 struct PreparedHeader {
     uint32_t magic, R, K, gd, slots;
@@ -47,6 +49,11 @@ struct StageParams {
     float scale;    // 2^k applied to residuals and codewords of this stage
     float a, b;     // |score error| <= a * ||Z|| + b
     float unsafe;   // non-zero: the scaled codebook left the half-precision range
+};
+
+struct StagePartial {
+    double max_norm2;   // largest squared norm among this part's codewords
+    float lo, hi;       // smallest and largest entry
 };
 
 struct StageMaxima {

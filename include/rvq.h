@@ -135,6 +135,22 @@ int rvq_encode(const rvq_config *cfg /* host */, const void *x, int64_t n, int64
                void *stream /* cudaStream_t */);
 
 /*
+ * Encode and, in the same pass, the EMA statistics of this batch (Section 3:
+ * the codebooks are learnt from the encoder's own assignments, batch after
+ * batch).  Results are those of rvq_encode followed by rvq_ema_stats on the
+ * codes it produced: the residual entering every stage is already in registers
+ * when its code is chosen, so x is not read and re-scaled a second time.
+ *   batch_count  out  float32 [R][K]             (overwritten)
+ *   batch_sum    out  float32 [R][K][group_dim]  (overwritten; 16-byte aligned)
+ *   workspace         rvq_workspace_bytes(cfg, n) bytes, 256-byte aligned
+ * Follow with rvq_ema_apply (after summing over devices, if several).
+ */
+int rvq_encode_stats(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
+                     const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+                     float *batch_count, float *batch_sum, void *workspace, size_t workspace_bytes,
+                     rvq_status *status, void *stream /* cudaStream_t */);
+
+/*
  * The same encode computed entirely in float32 on the CUDA cores (every
  * distance in the direct form sum((z - e)^2), no tensor cores, no prepared
  * operands).  Same arguments and results as rvq_encode; an order of magnitude

@@ -58,6 +58,8 @@ def _load() -> ctypes.CDLL:
     lib.rvq_encode.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.rvq_encode_exact.restype = ctypes.c_int
     lib.rvq_encode_exact.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp]
+    lib.rvq_encode_stats.restype = ctypes.c_int
+    lib.rvq_encode_stats.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.rvq_decode.restype = ctypes.c_int
     lib.rvq_decode.argtypes = [cfgp, vp, vp, i64, vp, vp, vp, i64, vp, vp]
     lib.rvq_ema_update.restype = ctypes.c_int
@@ -77,7 +79,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 
-EXPORTS = ("rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
+EXPORTS = ("rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
            "rvq_prepare_codebooks", "rvq_workspace_bytes", "rvq_encode", "rvq_decode",
            "rvq_ema_update")
 
@@ -140,6 +142,16 @@ def rvq_encode(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, wor
                         _stream(stream))
     if check:
         _check(rc, "rvq_encode")
+    return rc
+
+
+def rvq_encode_stats(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, batch_count, batch_sum,
+                     workspace, workspace_bytes, status=None, stream=None, check=True) -> int:
+    rc = lib.rvq_encode_stats(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
+                              _ptr(codes), _ptr(std_f16), _ptr(batch_count), _ptr(batch_sum), _ptr(workspace),
+                              workspace_bytes, _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_encode_stats")
     return rc
 
 

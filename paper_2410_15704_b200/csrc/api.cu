@@ -124,6 +124,38 @@ int rvq_encode(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_st
     return encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, stream, true);
 }
 
+int rvq_encode_stats(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                     const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+                     float *batch_count, float *batch_sum, void *workspace, size_t workspace_bytes,
+                     rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if (!batch_count || !batch_sum || !workspace) return RVQ_ERR_BADARG;
+    if (!aligned16(batch_sum) || !aligned256(workspace)) return RVQ_ERR_ALIGN;
+    if (workspace_bytes < ema_stats_scratch_bytes(s)) return RVQ_ERR_WORKSPACE;
+    if (!encode_tensor_supported(s)) {
+        // shapes without the fused kernel: encode, then the separate statistics pass
+        rc = encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, stream, true);
+        if (rc != RVQ_OK) return rc;
+        return launch_ema_stats(s, x, n, x_row_stride, codes, codebooks, batch_count, batch_sum, workspace,
+                                status, (cudaStream_t)stream);
+    }
+    if ((rc = check_rows(s, x, n, x_row_stride)) != RVQ_OK) return rc;
+    if (!codebooks || !prepared || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
+    if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    uint32_t *cnt = reinterpret_cast<uint32_t *>(workspace);
+    const int bins = s.R * s.K;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(cnt, 0, (size_t)bins * sizeof(uint32_t), st) != cudaSuccess ||
+        cudaMemsetAsync(batch_sum, 0, (size_t)bins * s.gd * sizeof(float), st) != cudaSuccess)
+        return RVQ_ERR_LAUNCH;
+    rc = launch_encode_tensor(s, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, st, cnt, batch_sum);
+    if (rc != RVQ_OK) return rc;
+    return launch_counts_to_float(cnt, batch_count, bins, st);
+}
+
 int rvq_encode_exact(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
                      const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
                      rvq_status *status, void *stream)

@@ -31,7 +31,8 @@ int launch_encode_scalar(const Shape &s, const void *x, int64_t n, int64_t strid
 bool encode_tensor_supported(const Shape &s);
 int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
                          const void *prepared, void *codes, uint16_t *std16, rvq_status *st,
-                         cudaStream_t stream);
+                         cudaStream_t stream, uint32_t *stat_cnt = nullptr, float *stat_sum = nullptr);
+int launch_counts_to_float(const uint32_t *cnt, float *out, int bins, cudaStream_t stream);
 int launch_decode_gather(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
                          const float *cb, void *out, int64_t stride, rvq_status *st,
                          cudaStream_t stream);

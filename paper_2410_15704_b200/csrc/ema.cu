@@ -143,6 +143,12 @@ int launch_ema_stats(const Shape &s, const void *x, int64_t n, int64_t stride, c
     return check_launch();
 }
 
+int launch_counts_to_float(const uint32_t *cnt, float *out, int bins, cudaStream_t stream)
+{
+    counts_to_float_kernel<<<(bins + 255) / 256, 256, 0, stream>>>(cnt, out, bins);
+    return check_launch();
+}
+
 int launch_ema_apply(const Shape &s, const float *batch_count, const float *batch_sum, float *cb,
                      float *ema_count, float *ema_sum, float decay, float eps, cudaStream_t stream)
 {

@@ -240,6 +240,8 @@ struct Params {
     uint16_t *std16;
     rvq_status *st;
     int tiles;          // 128-row tiles in the whole problem
+    uint32_t *stat_cnt; // optional EMA statistics of this batch: counts [R][K] ...
+    float *stat_sum;    // ... and sums of the stage inputs [R][K][32]; both null when not wanted
 };
 
 // The tiles of one CTA: a contiguous run, done in `rounds` rounds of nearly equal size (<= kTiles).
@@ -621,6 +623,17 @@ encode_tensor_kernel(const Params p)
                     }
                 }
                 if (deg) bj = 0;
+                if (p.stat_sum && valid) {
+                    // EMA statistics (Section 3): this row's stage input joins the bin of its code
+                    const size_t bin = (size_t)r * s.K + bj;
+                    atomicAdd(p.stat_cnt + bin, 1u);
+                    if (!deg) {
+                        float4 *m = reinterpret_cast<float4 *>(p.stat_sum + bin * 32);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            atomicAdd(m + q, make_float4(z[4 * q], z[4 * q + 1], z[4 * q + 2], z[4 * q + 3]));
+                    }
+                }
                 if (!deg) {
                     const float *ew = cbr + (size_t)bj * 32;
 #pragma unroll
@@ -693,7 +706,7 @@ bool encode_tensor_supported(const Shape &s)
 
 int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
                          const void *prepared, void *codes, uint16_t *std16, rvq_status *st,
-                         cudaStream_t stream)
+                         cudaStream_t stream, uint32_t *stat_cnt, float *stat_sum)
 {
     if (n == 0) return RVQ_OK;
     const int64_t rows = n * s.G;
@@ -705,7 +718,7 @@ int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t strid
         return RVQ_ERR_DEVICE;
     if (cudaFuncSetAttribute(encode_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
-    Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)tiles};
+    Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)tiles, stat_cnt, stat_sum};
     const int64_t groups = (tiles + kTiles - 1) / kTiles;
     const int grid = (int)(groups < sms ? groups : sms);
     encode_tensor_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);

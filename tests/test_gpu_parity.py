@@ -179,6 +179,29 @@ def test_tensor_encode_equals_exact_encode():
         assert st["wait_timeouts"] == 0 and st["exhaustive_rows"] < 1e-3 * rows
 
 
+def test_fused_encode_stats_equals_encode_then_stats():
+    """rvq_encode_stats gives rvq_encode's codes and rvq_ema_stats' counts and sums."""
+    for w in (rvq_synth.key_cache(tokens=700), rvq_synth.tiny(1000)):
+        cfg = config_of(w)
+        xd = x_to_device(w.x, cfg.x_dtype)
+        codes, std_bits, _, b = gpu_encode(cfg, xd, w.n, w.codebooks)
+        R, K, gd = w.codebooks.shape
+        c1, s1 = torch.empty(R, K, device="cuda"), torch.empty(R, K, gd, device="cuda")
+        rvq.rvq_ema_stats(cfg, xd, w.n, w.dim, b.codes, b.codebooks, c1, s1, b.workspace, b.workspace_bytes, b.status)
+        b2 = rvq.alloc_buffers(cfg, w.n, w.codebooks)
+        c2, s2 = torch.full((R, K), -1.0, device="cuda"), torch.full((R, K, gd), 9.0, device="cuda")
+        rvq.rvq_encode_stats(cfg, xd, w.n, w.dim, b2.codebooks, b2.prepared, b2.codes, b2.std, c2, s2,
+                             b2.workspace, b2.workspace_bytes, b2.status)
+        torch.cuda.synchronize()
+        assert np.array_equal(codes, codes_to_numpy(cfg, b2.codes, w.n))
+        assert torch.equal(c1, c2) and int(c2.sum().item()) == w.n * w.groups * R
+        scale = torch.clamp(c1, min=1.0)[..., None]
+        assert torch.max(torch.abs(s1 - s2) / scale).item() <= 1e-4
+        ref_cnt, ref_sum = oracle.ema_stats(w.x, codes, w.codebooks, w.layout)
+        assert np.array_equal(c2.cpu().numpy(), ref_cnt)
+        assert np.max(np.abs(s2.cpu().numpy() - ref_sum) / np.maximum(1.0, ref_cnt)[..., None]) <= RECON_TOL
+
+
 def test_tensor_encode_hostile_codebooks():
     """Codebooks far outside the half-precision range, duplicates and zeros: still exact."""
     g = np.random.default_rng(5)

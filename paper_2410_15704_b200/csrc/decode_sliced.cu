@@ -170,12 +170,15 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
             } else {
                 // Lane g holds element pairs (2c, 2c+1) of group g, i.e. channels 32 slice + 8c + g and + 4.
                 // Lane c' of the 4-lane set wants pairs c' of all four groups: a 4x4 transpose of words.
-#pragma unroll
-                for (int jx = 1; jx < 4; ++jx) {
-                    const int give = g ^ jx;                                 // the word the partner wants is w[partner]
-                    const uint32_t send = give == 0 ? w[0] : give == 1 ? w[1] : give == 2 ? w[2] : w[3];
-                    const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, send, jx);   // partner's w[g]: group (g ^ jx), pair g
-                    if (give == 0) w[0] = got; else if (give == 1) w[1] = got; else if (give == 2) w[2] = got; else w[3] = got;
+                // two butterfly steps: exchange odd/even words with lane g^1, then word pairs with lane g^2
+                {
+                    const bool b1 = g & 1, b2 = g & 2;
+                    const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w[0] : w[1], 1);
+                    const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w[2] : w[3], 1);
+                    if (b1) { w[0] = r0; w[2] = r1; } else { w[1] = r0; w[3] = r1; }
+                    const uint32_t r2 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[0] : w[2], 2);
+                    const uint32_t r3 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[1] : w[3], 2);
+                    if (b2) { w[0] = r2; w[1] = r3; } else { w[2] = r2; w[3] = r3; }
                 }
                 // now w[q] = pair g of group q: (element 2g of group q, element 2g+1 of group q)
                 const uint32_t o0 = __byte_perm(w[0], w[1], 0x5410), o1 = __byte_perm(w[2], w[3], 0x5410);

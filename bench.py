@@ -30,7 +30,14 @@ import numpy as np  # noqa: E402
 
 import rvq_synth  # noqa: E402
 
-WORKLOAD = "key_cache: 4096 tokens x 8 heads x 128 bf16, strided groups of 32, R=8, K=1024"
+def workload_name(tokens):
+    return f"key_cache: {tokens} tokens x 8 heads x 128 bf16, strided groups of 32, R=8, K=1024"
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one encode launch on the default workload, from the ncu
+# capture summarised in profiles/encode_tensor_key_cache.md (x 8.4 MB, codebooks and operand image 3.3 MB;
+# the 2.2 MB of outputs stay in L2).  Reported only for the workload and kernel it was taken on.
+ENCODE_DRAM_TRAFFIC = {4096: 11686144}
 METRIC = "RVQ hot path (encode+decode+EMA update) head vectors per second"
 UNIT = "Mvectors/s"
 L2_FLUSH_BYTES = 256 << 20
@@ -120,7 +127,7 @@ def run_reference(args):
         return
     import oracle
     oracle.build()
-    w = rvq_synth.key_cache()
+    w = rvq_synth.key_cache(tokens=args.tokens)
     # a bounded sample per step, sized from a calibration run so that all K steps take about 90 s
     t_cal = min(oracle_step(w, oracle, 512) for _ in range(max(1, args.warmup)))
     n_sample = int(min(w.n, max(64, 90.0 / max(1, args.steps) / (t_cal / 512))))
@@ -131,9 +138,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": f"first {n_sample} of 32768 head vectors per step"},
+        "data": "synthetic", "config": {"workload": workload_name(args.tokens), "sample": f"first {n_sample} of {w.n} head vectors per step"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-                         "sample": f"first {n_sample} of 32768 head vectors per step, {args.steps} steps"},
+                         "sample": f"first {n_sample} of {w.n} head vectors per step, {args.steps} steps"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -158,7 +165,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # every rank works on its own seeded batch of the same shape (weak scaling)
-    w = rvq_synth.key_cache(seed=1002 + rank)
+    w = rvq_synth.key_cache(tokens=args.tokens, seed=1002 + rank)
     base = rvq_synth.key_cache(tokens=8, seed=1002)      # shared initial codebooks
     w.codebooks = base.codebooks
     cfg = rvq.make_config(w.dim, w.group_dim, w.layout, w.depth, w.codebook_size, w.code_bits, rvq.BF16, 0)
@@ -286,7 +293,7 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32 (f16 tensor-core operands, f32 accumulate)", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "vectors_per_gpu": n, "l2": "flushed (256 MB write) before every timed step",
+        "config": {"workload": workload_name(args.tokens), "vectors_per_gpu": n, "l2": "flushed (256 MB write) before every timed step",
                    "timing": "CUDA events around each step on the launch stream, summed over K steps"},
         "phases": {
             "encode": {"ms": enc_ms, "Mvectors/s": n / enc_ms / 1e3, "TFLOP/s": enc_tflops,
@@ -297,7 +304,7 @@ def run_ours(args):
             "prepare": {"ms": statistics.mean(ev["prepare"])},
         },
         "roofline": {"kernel": "encode", "bound": "tensor", "achieved": enc_tflops, "peak": tensor_peak,
-                     "unit": "TFLOP/s", "frac": enc_tflops / tensor_peak, "traffic": None,
+                     "unit": "TFLOP/s", "frac": enc_tflops / tensor_peak, "traffic": ENCODE_DRAM_TRAFFIC.get(args.tokens),
                      "peak_source": f"{peaks['source']} bf16 burst x1 (f16 operands, same rate)"},
         "e2e": {"value": n * world * args.steps / (e2e_ms * 1e-3) / 1e6, "unit": UNIT,
                 "h2d_bytes_per_step": x_host.numel() * 2,
@@ -312,12 +319,13 @@ def run_ours(args):
         import oracle
         oracle.build()
         # the oracle as it stands on the host cores: whole batches until about 10 s have passed
-        t, reps = 0.0, 0
+        t, reps, n_cpu = 0.0, 0, min(n, 32768)
         while t < 10.0 and reps < 12:
-            t += oracle_step(w, oracle, n)
+            t += oracle_step(w, oracle, n_cpu)
             reps += 1
-        line["cpu_baseline"] = {"value": n * reps / t / 1e6, "unit": UNIT, "cores": oracle.threads(),
-                                "kind": "oracle", "sample": f"{reps} steps over all {n} head vectors ({t:.1f} s)"}
+        line["cpu_baseline"] = {"value": n_cpu * reps / t / 1e6, "unit": UNIT, "cores": oracle.threads(),
+                                "kind": "oracle",
+                                "sample": f"{reps} steps over the first {n_cpu} of {n} head vectors ({t:.1f} s)"}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -330,6 +338,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tokens", type=int, default=4096,
+                    help="tokens per GPU of the key-cache recipe (default: the quoted workload, 4096)")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps

@@ -1,0 +1,154 @@
+#!/usr/bin/env python
+"""Per-kernel timings of the residual-VQ library on one GPU, one JSON line per case.
+
+  python paper_2410_15704_b200/kernel_bench.py encode key_cache:4096 value_cache:32768 tiny:4096
+  python paper_2410_15704_b200/kernel_bench.py decode decode_bandwidth:131072
+  python paper_2410_15704_b200/kernel_bench.py ema ema_learning:131072
+
+A case is `<workload>:<tokens>` (workload names of `rvq_synth`; `tiny:<n>` takes a vector count).  Each
+launch is timed with CUDA events on the launching stream after three warm-up launches; before every timed
+launch a 256 MB buffer is written so that nothing of the inputs is left in L2.  `--reps N` launches are timed
+and the median and the best are printed.  Encode reports useful flops (2·group_dim·K·R·G per vector)
+against the dense bf16 peak, decode and EMA report algorithmic bytes against the copy bandwidth; both peaks
+come from MEASURED_PEAKS.json beside the package when it exists.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import paper_2410_15704_b200 as rvq  # noqa: E402
+import rvq_synth  # noqa: E402
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p["hbm_gbs"], p["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def make(spec, **kw):
+    name, count = spec.split(":")
+    w = rvq_synth.tiny(int(count)) if name == "tiny" else rvq_synth.WORKLOADS[name](int(count), **kw)
+    return name, w
+
+
+def timed(fn, reps, flush):
+    for _ in range(3):
+        fn()
+    ts = []
+    for _ in range(reps):
+        flush.fill_(1)
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        fn()
+        e.record()
+        torch.cuda.synchronize()
+        ts.append(s.elapsed_time(e))
+    return statistics.median(ts), min(ts)
+
+
+def config_of(w, bits=None):
+    dt = {"f32": rvq.F32, "bf16": rvq.BF16, "f16": rvq.F16}
+    return rvq.make_config(w.dim, w.group_dim, w.layout, w.depth, w.codebook_size,
+                           w.code_bits if bits is None else bits, dt[w.out_dtype if w.x is None else w.x_dtype], 0)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "ema"])
+    ap.add_argument("cases", nargs="+")
+    ap.add_argument("--reps", type=int, default=10)
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("kernel_bench.py needs a CUDA device: there is no CPU fallback")
+    hbm, tensor, src = peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    for spec in args.cases:
+        if args.kernel == "decode" and spec.startswith("decode_bandwidth"):
+            runs = [make(spec, layout=0), make(spec, layout=1)]
+        else:
+            runs = [make(spec)]
+        for name, w in runs:
+            n, G, R, K, gd = w.n, w.groups, w.depth, w.codebook_size, w.group_dim
+            code_b = (G * R * w.code_bits + 31) // 32 * 4
+            line = {"kernel": args.kernel, "workload": name, "vectors": n, "K": K, "R": R,
+                    "layout": "strided" if w.layout else "contiguous", "code_bits": w.code_bits}
+            if args.kernel == "decode":
+                cfg = config_of(w)
+                b = rvq.alloc_buffers(cfg, n, w.codebooks)
+                tdt = rvq.TORCH_DTYPE[cfg.x_dtype]
+                if getattr(w, "codes", None) is not None:
+                    codes, std_bits = w.codes, w.std_bits
+                else:   # a workload without stored codes: encode it first
+                    x = torch.from_numpy(w.x).to(tdt).cuda()
+                    rvq.rvq_encode(cfg, x, n, w.dim, b.codebooks, b.prepared, b.codes, b.std,
+                                   b.workspace, b.workspace_bytes, b.status)
+                    codes = std_bits = None
+                if codes is not None:
+                    cfg = config_of(w, bits=16)
+                    code_b = G * R * 2
+                    b = rvq.alloc_buffers(cfg, n, w.codebooks)
+                    b.codes.view(torch.int16)[: n * G * R].copy_(
+                        torch.from_numpy(codes.astype(np.uint16).view(np.int16).reshape(-1)))
+                    b.std.copy_(torch.from_numpy(std_bits.view(np.int16)))
+                out = torch.empty(n, w.dim, dtype=tdt, device="cuda")
+                med, best = timed(lambda: rvq.rvq_decode(cfg, b.codes, b.std, n, b.codebooks, b.prepared, out,
+                                                         w.dim, b.status), args.reps, flush)
+                nbytes = n * (code_b + 2 + w.dim * out.element_size())
+                line.update(ms_median=med, ms_best=best, bytes=nbytes, GBps=nbytes / med / 1e6,
+                            frac_hbm=nbytes / med / 1e6 / hbm, peak=hbm, peak_source=src)
+            else:
+                cfg = config_of(w)
+                b = rvq.alloc_buffers(cfg, n, w.codebooks)
+                x = torch.from_numpy(w.x).to(rvq.TORCH_DTYPE[cfg.x_dtype]).cuda()
+                bc = torch.empty(R, K, device="cuda")
+                bs = torch.empty(R, K, gd, device="cuda")
+                if args.kernel == "encode":
+                    fn = lambda: rvq.rvq_encode(cfg, x, n, w.dim, b.codebooks, b.prepared, b.codes, b.std,
+                                                b.workspace, b.workspace_bytes, b.status)
+                elif args.kernel == "encode_exact":
+                    fn = lambda: rvq.rvq_encode_exact(cfg, x, n, w.dim, b.codebooks, b.prepared, b.codes, b.std,
+                                                      b.status)
+                elif args.kernel == "encode_stats":
+                    fn = lambda: rvq.rvq_encode_stats(cfg, x, n, w.dim, b.codebooks, b.prepared, b.codes, b.std,
+                                                      bc, bs, b.workspace, b.workspace_bytes, b.status)
+                else:
+                    rvq.rvq_encode(cfg, x, n, w.dim, b.codebooks, b.prepared, b.codes, b.std,
+                                   b.workspace, b.workspace_bytes, b.status)
+                    fn = lambda: rvq.rvq_ema_stats(cfg, x, n, w.dim, b.codes, b.codebooks, bc, bs,
+                                                   b.workspace, b.workspace_bytes, b.status)
+                med, best = timed(fn, args.reps, flush)
+                if args.kernel == "ema":
+                    nbytes = n * (w.dim * x.element_size() + code_b) + 2 * R * K * (gd + 1) * 4
+                    line.update(ms_median=med, ms_best=best, bytes=nbytes, GBps=nbytes / med / 1e6,
+                                frac_hbm=nbytes / med / 1e6 / hbm, peak=hbm, peak_source=src)
+                else:
+                    flops = 2.0 * gd * K * R * G * n
+                    st = rvq.read_status(b.status)
+                    line.update(ms_median=med, ms_best=best, Mvectors_per_s=n / med / 1e3,
+                                useful_TFLOPs=flops / med / 1e9, frac_tensor=flops / med / 1e9 / tensor,
+                                peak=tensor, peak_source=src,
+                                rescored_rows_per_launch=st["rescored_rows"] // (args.reps + 3),
+                                exhaustive_rows=st["exhaustive_rows"], wait_timeouts=st["wait_timeouts"])
+            print(json.dumps(line), flush=True)
+            del b
+            torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()

@@ -174,7 +174,7 @@ int rvq_decode(const rvq_config *cfg, const void *codes, const uint16_t *std_f16
     if (!codebooks || !prepared || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
     if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
     if (decode_sliced_supported(s))
-        return launch_decode_sliced(s, codes, std_f16, n, prepared, x_out, out_row_stride, status, (cudaStream_t)stream);
+        return launch_decode_sliced(s, codes, std_f16, n, codebooks, prepared, x_out, out_row_stride, status, (cudaStream_t)stream);
     return launch_decode_gather(s, codes, std_f16, n, codebooks, x_out, out_row_stride, status, (cudaStream_t)stream);
 }
 

@@ -4,19 +4,24 @@
 // Every output element needs one codeword element per stage, so a head vector of
 // 256 output bytes gathers 1024 table entries: the gather, not HBM, is the
 // limit, and it has to come from shared memory without bank conflicts.
-//   - A CTA keeps one channel slice (8 of the 32 codeword channels) of all
-//     stages as 15-bit levels: 128 bytes per code = 8 stages x 16 bytes.  The
-//     four slices of a row tile are handled by four CTAs; the codes they share
-//     come from L2.
-//   - One thread produces the 8 channels of one (group row, slice).  It reads
-//     its 8 codes as one 16-byte load and visits the stages in an order rotated
-//     by its lane, so the 8 lanes of a quarter warp always touch 8 different
-//     16-byte bank groups whatever the codes are.
+//   - A CTA keeps one channel slice (CH = 8 of the 32 codeword channels, 4 when
+//     there are more than 1536 codes per stage) of all stages as 15-bit levels:
+//     16 CH bytes per code = 8 stages x 2 CH bytes.  The 32 / CH slices of a row
+//     tile are handled by as many CTAs; the codes they share come from L2.
+//   - One thread produces the CH channels of one (group row, slice).  It reads
+//     its 8 codes as one 16-byte load (or unpacks them from the bit stream) and
+//     visits the stages in an order rotated by its lane, so with CH = 8 the 8
+//     lanes of a quarter warp always touch 8 different 16-byte bank groups
+//     whatever the codes are (with CH = 4 two lanes of a half warp can meet).
 //   - A level q becomes the float 1 + q 2^-15 by one byte permute (the stored
 //     level carries the exponent's low bit), and one packed float32x2 FMA with
 //     the stage's step adds two channels to their float32 sums, which start at
 //     the affine offset of all stages; the sums are then multiplied by the
 //     stored deviation and rounded once.
+//   - The level tables are off by at most dp->err (half a level per stage) times
+//     the deviation.  A row whose deviation makes that more than 0.9e-3 sums the
+//     float32 codewords instead (stage order, from global memory), so the result
+//     before the output rounding is always within 1e-3 of the exact sum.
 //   - With strided groups the 4 lanes of a head vector exchange their results so
 //     that every lane stores 16 contiguous bytes.
 #include "prepared.cuh"
@@ -62,26 +67,30 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
     return d;
 }
 
-template <int DT>
+template <int DT, int CH>
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
-                     const uint8_t *__restrict__ dsec, void *__restrict__ out, int64_t stride, rvq_status *st)
+                     const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
+                     int64_t stride, rvq_status *st)
 {
-    extern __shared__ __align__(128) uint8_t table[];            // [K][8 stages][16 bytes]
+    extern __shared__ __align__(128) uint8_t table[];            // [K][8 stages][2 CH bytes]
+    constexpr int NS = 32 / CH;                                  // slices
+    constexpr uint32_t kEntry = 2 * CH, kLine = 16 * CH;         // bytes per (code, stage) and per code
     const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
-    const int slice = blockIdx.x & 3, part = blockIdx.x >> 2, parts = gridDim.x >> 2;
+    const int slice = blockIdx.x % NS, part = blockIdx.x / NS, parts = gridDim.x / NS;
     const int tid = threadIdx.x, lane = tid & 31, rot = lane & 7;
     {
-        const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256) + (size_t)slice * s.K * 8;
+        const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256) + (size_t)slice * s.K * CH;
         uint4 *dst = reinterpret_cast<uint4 *>(table);
-        for (int t = tid; t < s.K * 8; t += kDecThreads) dst[t] = __ldg(src + t);
+        for (int t = tid; t < s.K * CH; t += kDecThreads) dst[t] = __ldg(src + t);
     }
     // this thread visits stage (rot + k) & 7 at step k: its steps' scales and line offsets
     float step[8];
     uint32_t unit[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { step[k] = dp->step[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * 16u; }
+    for (int k = 0; k < 8; ++k) { step[k] = dp->step[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * kEntry; }
     const float bias = dp->bias;
+    const float exact_above = dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY;   // deviations the tables may serve
     __syncthreads();
 
     const int64_t rows = n * 4;
@@ -97,12 +106,27 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
             if (s.bits == 16 && s.R == 8) {
                 const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + row);
                 cw[0] = c.x; cw[1] = c.y; cw[2] = c.z; cw[3] = c.w;
+            } else if (s.bits == 11 && s.R == 8) {
+                // 88 bits starting at bit 88 g of the vector's 352: a window of up to four words
+                const uint32_t *wv = reinterpret_cast<const uint32_t *>(codes) + v * 11;
+                const int wi = (g * 88) >> 5, sh = (g * 88) & 31;
+                const uint32_t q0 = __ldg(wv + wi), q1 = __ldg(wv + wi + 1), q2 = __ldg(wv + wi + 2);
+                const uint32_t q3 = wi + 3 < 11 ? __ldg(wv + wi + 3) : 0u;
+                const uint32_t u0 = __funnelshift_r(q0, q1, sh), u1 = __funnelshift_r(q1, q2, sh);
+                const uint32_t u2 = __funnelshift_r(q2, q3, sh);
+                // codes at bits 0, 11, ..., 77 of u0:u1:u2
+                const uint32_t c0 = u0 & 0x7FFu, c1 = (u0 >> 11) & 0x7FFu;
+                const uint32_t c2 = __funnelshift_r(u0, u1, 22) & 0x7FFu, c3 = (u1 >> 1) & 0x7FFu;
+                const uint32_t c4 = (u1 >> 12) & 0x7FFu, c5 = __funnelshift_r(u1, u2, 23) & 0x7FFu;
+                const uint32_t c6 = (u2 >> 2) & 0x7FFu, c7 = (u2 >> 13) & 0x7FFu;
+                cw[0] = c0 | (c1 << 16); cw[1] = c2 | (c3 << 16); cw[2] = c4 | (c5 << 16); cw[3] = c6 | (c7 << 16);
             } else {
                 const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes;
                 for (int r = 0; r < s.R; ++r)
                     cw[r >> 1] |= read_code(vec, g * s.R + r, s.bits, s.code_bytes) << (16 * (r & 1));
             }
         }
+        const uint32_t cn[4] = {cw[0], cw[1], cw[2], cw[3]};      // natural order, for the exact route
         // rotate the 8 halves left by `rot` so that step k finds its code at a fixed place
         {
             uint32_t a0 = cw[0], a1 = cw[1], a2 = cw[2], a3 = cw[3];
@@ -129,74 +153,122 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
             }
         }
         // two channels per packed float32x2 accumulator, started at the affine offset
-        float2 acc[4];
+        float2 acc[CH / 2];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[i] = make_float2(bias, bias);
+        for (int i = 0; i < CH / 2; ++i) acc[i] = make_float2(bias, bias);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
-            const uint4 e = *reinterpret_cast<const uint4 *>(table + j * 128u + unit[k]);
             const float2 sk = make_float2(step[k], step[k]);
-            acc[0] = fma2(make_float2(level_to_float<0>(e.x), level_to_float<1>(e.x)), sk, acc[0]);
-            acc[1] = fma2(make_float2(level_to_float<0>(e.y), level_to_float<1>(e.y)), sk, acc[1]);
-            acc[2] = fma2(make_float2(level_to_float<0>(e.z), level_to_float<1>(e.z)), sk, acc[2]);
-            acc[3] = fma2(make_float2(level_to_float<0>(e.w), level_to_float<1>(e.w)), sk, acc[3]);
+            uint32_t e[CH / 2];
+            if (CH == 8) {
+                const uint4 t = *reinterpret_cast<const uint4 *>(table + j * kLine + unit[k]);
+                e[0] = t.x; e[1] = t.y; e[CH / 2 - 2] = t.z; e[CH / 2 - 1] = t.w;
+            } else {
+                const uint2 t = *reinterpret_cast<const uint2 *>(table + j * kLine + unit[k]);
+                e[0] = t.x; e[1] = t.y;
+            }
+#pragma unroll
+            for (int i = 0; i < CH / 2; ++i)
+                acc[i] = fma2(make_float2(level_to_float<0>(e[i]), level_to_float<1>(e[i])), sk, acc[i]);
         }
         const float sd = live ? __half2float(__ushort_as_half(std16[v])) : 0.0f;
-        float o8[8];
+        float o8[CH];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { o8[2 * i] = acc[i].x * sd; o8[2 * i + 1] = acc[i].y * sd; }
+        for (int i = 0; i < CH / 2; ++i) { o8[2 * i] = acc[i].x * sd; o8[2 * i + 1] = acc[i].y * sd; }
+        if (fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
+            // too coarse for this deviation: the float32 codewords themselves, summed in stage order
+            float ex[CH];
+#pragma unroll
+            for (int i = 0; i < CH; ++i) ex[i] = 0.0f;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                if (r < s.R) {
+                    uint32_t j = (r & 1) ? (cn[r >> 1] >> 16) : (cn[r >> 1] & 0xFFFFu);
+                    if (j >= (uint32_t)s.K) j = 0;
+                    const float4 *e = reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * 32 + slice * CH);
+#pragma unroll
+                    for (int q = 0; q < CH / 4; ++q) {
+                        const float4 t = __ldg(e + q);
+                        ex[4 * q] += t.x; ex[4 * q + 1] += t.y; ex[4 * q + 2] += t.z; ex[4 * q + 3] += t.w;
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < CH; ++i) o8[i] = ex[i] * sd;
+        }
 
         if (DT == RVQ_F32) {
             if (s.layout == RVQ_GROUP_CONTIGUOUS) {
                 if (live) {
-                    float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + v * stride + g * 32 + slice * 8);
-                    o[0] = make_float4(o8[0], o8[1], o8[2], o8[3]);
-                    o[1] = make_float4(o8[4], o8[5], o8[6], o8[7]);
+                    float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + v * stride + g * 32 + slice * CH);
+#pragma unroll
+                    for (int i = 0; i < CH / 4; ++i)
+                        o[i] = make_float4(o8[4 * i], o8[4 * i + 1], o8[4 * i + 2], o8[4 * i + 3]);
                 }
             } else if (live) {
-                float *o = reinterpret_cast<float *>(out) + v * stride + slice * 32 + g;
+                float *o = reinterpret_cast<float *>(out) + v * stride + slice * CH * 4 + g;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) o[4 * i] = o8[i];         // channel (8 slice + i) * 4 + g
+                for (int i = 0; i < CH; ++i) o[4 * i] = o8[i];        // channel (CH slice + i) * 4 + g
             }
         } else {
-            uint32_t w[4];
+            uint32_t w[CH / 2];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) w[c] = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(o8[2 * c], o8[2 * c + 1]);
+            for (int c = 0; c < CH / 2; ++c) w[c] = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(o8[2 * c], o8[2 * c + 1]);
+            uint16_t *o16 = reinterpret_cast<uint16_t *>(out) + v * stride;
             if (s.layout == RVQ_GROUP_CONTIGUOUS) {
-                if (live)
-                    *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(out) + v * stride + g * 32 + slice * 8) =
-                        make_uint4(w[0], w[1], w[2], w[3]);
-            } else {
+                if (live) {
+                    if (CH == 8)
+                        *reinterpret_cast<uint4 *>(o16 + g * 32 + slice * 8) = make_uint4(w[0], w[1], w[CH / 2 - 2], w[CH / 2 - 1]);
+                    else
+                        *reinterpret_cast<uint2 *>(o16 + g * 32 + slice * 4) = make_uint2(w[0], w[1]);
+                }
+            } else if (CH == 8) {
                 // Lane g holds element pairs (2c, 2c+1) of group g, i.e. channels 32 slice + 8c + g and + 4.
                 // Lane c' of the 4-lane set wants pairs c' of all four groups: a 4x4 transpose of words.
                 // two butterfly steps: exchange odd/even words with lane g^1, then word pairs with lane g^2
+                uint32_t &w0 = w[0], &w1 = w[1], &w2 = w[CH / 2 - 2], &w3 = w[CH / 2 - 1];
                 {
                     const bool b1 = g & 1, b2 = g & 2;
-                    const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w[0] : w[1], 1);
-                    const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w[2] : w[3], 1);
-                    if (b1) { w[0] = r0; w[2] = r1; } else { w[1] = r0; w[3] = r1; }
-                    const uint32_t r2 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[0] : w[2], 2);
-                    const uint32_t r3 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[1] : w[3], 2);
-                    if (b2) { w[0] = r2; w[1] = r3; } else { w[2] = r2; w[3] = r3; }
+                    const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w0 : w1, 1);
+                    const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w2 : w3, 1);
+                    if (b1) { w0 = r0; w2 = r1; } else { w1 = r0; w3 = r1; }
+                    const uint32_t r2 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w0 : w2, 2);
+                    const uint32_t r3 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w1 : w3, 2);
+                    if (b2) { w0 = r2; w1 = r3; } else { w2 = r2; w3 = r3; }
                 }
                 // now w[q] = pair g of group q: (element 2g of group q, element 2g+1 of group q)
-                const uint32_t o0 = __byte_perm(w[0], w[1], 0x5410), o1 = __byte_perm(w[2], w[3], 0x5410);
-                const uint32_t o2 = __byte_perm(w[0], w[1], 0x7632), o3 = __byte_perm(w[2], w[3], 0x7632);
+                const uint32_t o0 = __byte_perm(w0, w1, 0x5410), o1 = __byte_perm(w2, w3, 0x5410);
+                const uint32_t o2 = __byte_perm(w0, w1, 0x7632), o3 = __byte_perm(w2, w3, 0x7632);
                 // channels 32 slice + 8 g + 0..7: element 2g of groups 0..3, then element 2g+1 of groups 0..3
+                if (live) *reinterpret_cast<uint4 *>(o16 + slice * 32 + g * 8) = make_uint4(o0, o1, o2, o3);
+            } else {
+                // Lane g holds elements 4 slice + 0..3 of group g as w[0] = (e0, e1), w[1] = (e2, e3); the
+                // 16 channels 16 slice .. 16 slice + 15 are element-major, so lane L stores element L of
+                // the four groups.  Exchange words with lane g^2, then halves with lane g^1.
+                const bool b1 = g & 1, b2 = g & 2;
+                const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[0] : w[1], 2);
+                // lanes 0, 1 now hold (e0, e1) of groups g and g + 2; lanes 2, 3 hold (e2, e3) of g - 2 and g
+                const uint32_t lo_g = b2 ? r0 : w[0], hi_g = b2 ? w[1] : r0;   // lower and upper group of the pair
+                // keep the half this lane stores (e_L), send the other one
+                const uint32_t keep = __byte_perm(lo_g, hi_g, b1 ? 0x7632 : 0x5410);
+                const uint32_t send = __byte_perm(lo_g, hi_g, b1 ? 0x5410 : 0x7632);
+                const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+                // keep = element L of groups (g & 1) and (g & 1) + 2, got = element L of the other two
+                const uint32_t even = b1 ? got : keep, odd = b1 ? keep : got;   // groups (0, 2) and (1, 3)
                 if (live)
-                    *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(out) + v * stride + slice * 32 + g * 8) =
-                        make_uint4(o0, o1, o2, o3);
+                    *reinterpret_cast<uint2 *>(o16 + slice * 16 + g * 4) =
+                        make_uint2(__byte_perm(even, odd, 0x5410), __byte_perm(even, odd, 0x7632));
             }
         }
     }
-    if (bad && st) atomicAdd(&st->bad_codes, bad);
+    if (bad && st && slice == 0) atomicAdd(&st->bad_codes, bad);   // every slice sees the same codes
 }
 
 }  // namespace
 
 int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
-                         const void *prepared, void *out, int64_t stride, rvq_status *st,
+                         const float *cb, const void *prepared, void *out, int64_t stride, rvq_status *st,
                          cudaStream_t stream)
 {
     if (n == 0) return RVQ_OK;
@@ -206,21 +278,29 @@ int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std1
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return RVQ_ERR_DEVICE;
-    const size_t smem = (size_t)s.K * 128;
+    const int ch = decode_slice_channels(s.K), ns = 32 / ch;
+    const size_t smem = (size_t)s.K * 16 * ch;
     const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
-    int parts = sms / 4;
+    int parts = sms / ns;
     if (parts > tiles) parts = (int)tiles;
     if (parts < 1) parts = 1;
     auto launch = [&](auto kernel) -> int {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return RVQ_ERR_LAUNCH;
-        kernel<<<parts * 4, kDecThreads, smem, stream>>>(s, codes, std16, n, p + off, out, stride, st);
+        kernel<<<parts * ns, kDecThreads, smem, stream>>>(s, codes, std16, n, p + off, cb, out, stride, st);
         return check_launch();
     };
+    if (ch == 8) {
+        switch (s.dtype) {
+        case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32, 8>);
+        case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16, 8>);
+        default: return launch(decode_sliced_kernel<RVQ_F16, 8>);
+        }
+    }
     switch (s.dtype) {
-    case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32>);
-    case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16>);
-    default: return launch(decode_sliced_kernel<RVQ_F16>);
+    case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32, 4>);
+    case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16, 4>);
+    default: return launch(decode_sliced_kernel<RVQ_F16, 4>);
     }
 }
 

@@ -23,18 +23,21 @@ struct PreparedHeader {
 
 // Decoder section (group_dim 32, R <= 8, K <= kDecodeMaxK): per stage an affine
 // map value = lo + (f - 1) * step with f = 1 + q * 2^-15 in [1, 2) the float whose
-// mantissa bits 22..8 are the 15-bit level q, then four channel slices of the
-// codebooks as levels: table[slice][code][stage 0..7][8 channels] uint16, each
-// with bit 15 set (it becomes the lowest exponent bit of f).
+// mantissa bits 22..8 are the 15-bit level q, then channel slices of the
+// codebooks as levels: table[slice][code][stage 0..7][CH channels] uint16, each
+// with bit 15 set (it becomes the lowest exponent bit of f).  A slice is CH = 8
+// channels wide (four slices) while K <= kDecodeWideK and 4 channels (eight
+// slices) above, so that one slice of all codes fits the shared memory of a CTA.
 struct DecodeParams {
     float step[8];    // (max - min) * 32768 / 32767 per stage, 0 for absent stages
     float bias;       // sum over stages of (min - step)
     float err;        // bound on |sum of table values - sum of float32 values| per channel
     float pad[6];
 };
-constexpr int kDecodeMaxK = 1536;                         // 128 bytes per code per slice in shared memory
-constexpr int kDecodeSlices = 4;
-__host__ __device__ inline size_t decode_table_bytes(int K) { return (size_t)kDecodeSlices * K * 128; }
+constexpr int kDecodeWideK = 1536;                        // 128 bytes per code per slice in shared memory
+constexpr int kDecodeMaxK = 3072;                         // 64 bytes per code per slice
+__host__ __device__ inline int decode_slice_channels(int K) { return K <= kDecodeWideK ? 8 : 4; }
+__host__ __device__ inline size_t decode_table_bytes(int K) { return (size_t)K * 512; }   // 32 channels x 8 stages x 2 bytes
 __host__ __device__ inline bool decode_sliced_supported(const Shape &s)
 {
     // 16-bit outputs only: their own rounding (2^-9 or 2^-12 relative) dwarfs the table's

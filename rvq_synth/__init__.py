@@ -75,12 +75,17 @@ def laplace(seed: int, count: int) -> np.ndarray:
 
 
 def randint(seed: int, count: int, high: int) -> np.ndarray:
-    """``count`` integers uniform on ``[0, high)`` (``high`` a power of two)."""
-    assert high & (high - 1) == 0
+    """``count`` integers uniform on ``[0, high)``: bits 20.. of the draw when
+    ``high`` is a power of two, else the top 32 bits scaled by ``high``."""
+    assert 0 < high < (1 << 31)
     out = np.empty(count, dtype=np.int64)
     for lo in range(0, count, _CHUNK):
         m = min(_CHUNK, count - lo)
-        out[lo:lo + m] = (splitmix64(seed, lo, m) >> np.uint64(20)).astype(np.int64) & (high - 1)
+        draw = splitmix64(seed, lo, m)
+        if high & (high - 1) == 0:
+            out[lo:lo + m] = (draw >> np.uint64(20)).astype(np.int64) & (high - 1)
+        else:
+            out[lo:lo + m] = (((draw >> np.uint64(32)) * np.uint64(high)) >> np.uint64(32)).astype(np.int64)
     return out
 
 

@@ -77,6 +77,40 @@ def test_decode_bandwidth_full_size(layout):
     print(f"decode layout {layout}: bf16 max-abs {err:.2e}, fp32 max-abs {err32:.2e}")
 
 
+@pytest.mark.parametrize("K,bits,layout,dtype", [
+    (2048, 11, rvq_synth.CONTIGUOUS, "bf16"), (2048, 11, rvq_synth.STRIDED, "bf16"),
+    (2048, 16, rvq_synth.STRIDED, "f16"), (1537, 11, rvq_synth.CONTIGUOUS, "f16"),
+    (3072, 12, rvq_synth.STRIDED, "bf16"), (1536, 11, rvq_synth.STRIDED, "bf16"),
+    (3073, 12, rvq_synth.CONTIGUOUS, "bf16"),
+])
+def test_decode_large_codebooks(K, bits, layout, dtype):
+    """More than 1536 codes per stage: narrow table slices (up to 3072 codes), gathers beyond."""
+    w = rvq_synth.decode_bandwidth(tokens=1111, size=K, layout=layout)      # 8888 vectors: ragged tiles
+    cfg = rvq.make_config(w.dim, w.group_dim, layout, w.depth, K, bits, DT[dtype], 0)
+    got, st = gpu_decode(cfg, w.codes, w.std_bits, w.codebooks, w.n)
+    err = assert_recon_match(got, w.codes, w.std_bits, w.codebooks, w.dim, layout, cfg.x_dtype)
+    assert st["bad_codes"] == 0
+    print(f"decode K={K} bits={bits} layout={layout} {dtype}: max-abs {err:.2e}")
+
+
+@pytest.mark.parametrize("K,layout", [(1024, rvq_synth.CONTIGUOUS), (2048, rvq_synth.STRIDED)])
+def test_decode_large_deviations_take_the_exact_route(K, layout):
+    """Rows whose deviation would scale the level tables' error past 1e-3 sum float32 codewords."""
+    w = rvq_synth.decode_bandwidth(tokens=700, size=K, layout=layout)
+    sd = oracle.f16_value(w.std_bits)
+    sd[::3] *= 64.0                                     # table error would be ~1e-2 on these rows
+    sd[1::7] = 0.0
+    std_bits = oracle.f16_bits(sd)
+    cfg = rvq.make_config(w.dim, w.group_dim, layout, w.depth, K, 16, rvq.BF16, 0)
+    got, st = gpu_decode(cfg, w.codes, std_bits, w.codebooks, w.n)
+    # bf16's own rounding hides the difference on large values, so look at the small ones too
+    ref = oracle.decode(w.codes, std_bits, w.codebooks, w.dim, layout)
+    small = np.abs(ref) < 0.25
+    assert small[::3].sum() > 1000
+    assert np.all(np.abs(got - ref)[small] <= RECON_TOL + 2.0 ** -8 * np.abs(ref[small]))
+    assert_recon_match(got, w.codes, std_bits, w.codebooks, w.dim, layout, cfg.x_dtype)
+
+
 def test_decode_head_major_tiles():
     """Output rows written through a row stride: [head][token][dim] tiles."""
     w = rvq_synth.decode_bandwidth(tokens=1024)

@@ -392,10 +392,40 @@ encode_tensor_kernel(const Params p)
             const int g = (int)(grow - v * G);
             const bool valid = v < p.n;
 
+            // The warp's 32 / G head vectors (1024 elements) come in as 16-byte pieces through the
+            // warp's share of the parking area: word k sits at [k / 32][k % 32], and piece c of
+            // vector vl at position c ^ (vl mod 8) of its vector so that the reads below spread over the banks.
             float z[32];
+            {
+                const int eb = s.elem_bytes, ppv = s.dim * eb / 16;          // pieces per vector (>= 4)
+                const int64_t v_first = (row0 + q4 * 32) / G;
+                float *scr = reinterpret_cast<float *>(smem + kOffZ) + (rloc - lane);
+                for (int c = lane; c < (32 / G) * ppv; c += 32) {
+                    const int vl = c / ppv, off = c - vl * ppv;
+                    const int64_t vv = v_first + vl;
+                    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                    if (vv < p.n)
+                        val = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(p.x) + vv * p.stride * eb) + off);
+                    const int k = (vl * ppv + (off ^ (vl & 7 & (ppv - 1)))) * 4;
+                    *reinterpret_cast<uint4 *>(scr + (k >> 5) * kRowsPerPass + (k & 31)) = val;
+                }
+                __syncwarp();
+                const int vl = lane / G, sw = vl & 7 & (ppv - 1);
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-                z[i] = valid ? load_as_float(p.x, v * p.stride + channel_of(s.layout, G, 32, g, i), s.dtype) : 0.0f;
+                for (int i = 0; i < 32; ++i) {
+                    const int b = channel_of(s.layout, G, 32, g, i) * eb;      // byte within the vector
+                    const int k = (vl * ppv + ((b >> 4) ^ sw)) * 4 + ((b & 15) >> 2);
+                    const uint32_t word = __float_as_uint(scr[(k >> 5) * kRowsPerPass + (k & 31)]);
+                    float val;
+                    if (s.dtype == RVQ_F32) val = __uint_as_float(word);
+                    else {
+                        const uint16_t h = (b & 2) ? (uint16_t)(word >> 16) : (uint16_t)(word & 0xFFFFu);
+                        val = s.dtype == RVQ_BF16 ? __uint_as_float((uint32_t)h << 16) : __half2float(__ushort_as_half(h));
+                    }
+                    z[i] = valid ? val : 0.0f;
+                }
+                __syncwarp();
+            }
             // deviation over the G lanes of this head vector, same summation order as the scalar kernel
             float dev;
             {
@@ -479,31 +509,31 @@ encode_tensor_kernel(const Params p)
                     ++chunk_use;
                     if (!ok) break;
                     tc_fence_after();
-                    // four 32-column blocks; the next block loads while the current one is reduced
+                    // Four 32-column blocks.  Only the cell minima of a block are taken between two
+                    // loads, so that the accumulator is handed back to the MMA issuer as early as
+                    // possible; the rest of the reduction runs while the next chain computes.
                     uint32_t ua[32], ub[32];
-                    float ta[11], tb[11];
+                    float t0[11], t1[11], t2[11], t3[11];
                     tmem_ld32_issue(taddr, ua);
                     tmem_ld_wait(ua);
                     tmem_ld32_issue(taddr + 32, ub);
-                    const float ca0 = block_cells(ua, ta);
-                    list_block(w, ca0, c * 4, list_v, list_i, kRowsPerPass);
+                    const float c0 = block_cells(ua, t0);
                     tmem_ld_wait(ub);
                     tmem_ld32_issue(taddr + 64, ua);
-                    const float cb0 = block_cells(ub, tb);
-#pragma unroll
-                    for (int q = 0; q < 11; ++q) w.d[q] = min3(w.d[q], ta[q], tb[q]);
-                    list_block(w, cb0, c * 4 + 1, list_v, list_i, kRowsPerPass);
+                    const float c1 = block_cells(ub, t1);
                     tmem_ld_wait(ua);
                     tmem_ld32_issue(taddr + 96, ub);
-                    const float ca1 = block_cells(ua, ta);
-                    list_block(w, ca1, c * 4 + 2, list_v, list_i, kRowsPerPass);
+                    const float c2 = block_cells(ua, t2);
                     tmem_ld_wait(ub);
                     tc_fence_before();
                     mbar_arrive(BAR(kBarAccFree + tile));        // the accumulator may be overwritten
-                    const float cb1 = block_cells(ub, tb);
+                    const float c3 = block_cells(ub, t3);
 #pragma unroll
-                    for (int q = 0; q < 11; ++q) w.d[q] = min3(w.d[q], ta[q], tb[q]);
-                    list_block(w, cb1, c * 4 + 3, list_v, list_i, kRowsPerPass);
+                    for (int q = 0; q < 11; ++q) w.d[q] = fminf(min3(w.d[q], t0[q], t1[q]), fminf(t2[q], t3[q]));
+                    list_block(w, c0, c * 4, list_v, list_i, kRowsPerPass);
+                    list_block(w, c1, c * 4 + 1, list_v, list_i, kRowsPerPass);
+                    list_block(w, c2, c * 4 + 2, list_v, list_i, kRowsPerPass);
+                    list_block(w, c3, c * 4 + 3, list_v, list_i, kRowsPerPass);
                 }
                 if (!ok) break;
                 // take the residual back

@@ -67,19 +67,32 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
     return d;
 }
 
-template <int DT, int CH>
-__global__ void __launch_bounds__(kDecThreads, 1)
-decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
-                     const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
-                     int64_t stride, rvq_status *st)
+// F32T: the tables hold the float32 codebook entries themselves (16 bytes per stage with
+// CH = 4: the same shared-memory geometry as the 15-bit tables with CH = 8) and the sums are
+// exact float32 sums; otherwise 15-bit levels as described above.
+template <int DT, int CH, bool F32T>
+__device__ __forceinline__ void
+decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                   const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
+                   int64_t stride, rvq_status *st, uint8_t *table)
 {
-    extern __shared__ __align__(128) uint8_t table[];            // [K][8 stages][2 CH bytes]
+    // table: [K][8 stages][kEntry bytes] in shared memory
     constexpr int NS = 32 / CH;                                  // slices
-    constexpr uint32_t kEntry = 2 * CH, kLine = 16 * CH;         // bytes per (code, stage) and per code
+    if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;   // (a grid sized for another slice count)
+    constexpr uint32_t kEntry = (F32T ? 4 : 2) * CH, kLine = 8 * kEntry;   // bytes per (code, stage) and per code
     const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
     const int slice = blockIdx.x % NS, part = blockIdx.x / NS, parts = gridDim.x / NS;
     const int tid = threadIdx.x, lane = tid & 31, rot = lane & 7;
-    {
+    if (F32T) {
+        // entry (code j, stage r) = channels CH slice .. CH slice + CH - 1 of codeword j of stage r
+        for (int t = tid; t < s.K * 8; t += kDecThreads) {
+            const int r = t / s.K, j = t - r * s.K;
+            float *dst = reinterpret_cast<float *>(table + (size_t)j * kLine + r * kEntry);
+            const float *src = cb + ((size_t)r * s.K + j) * 32 + slice * CH;
+#pragma unroll
+            for (int i = 0; i < CH; ++i) dst[i] = r < s.R ? __ldg(src + i) : 0.0f;
+        }
+    } else {
         const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256) + (size_t)slice * s.K * CH;
         uint4 *dst = reinterpret_cast<uint4 *>(table);
         for (int t = tid; t < s.K * CH; t += kDecThreads) dst[t] = __ldg(src + t);
@@ -88,9 +101,9 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
     float step[8];
     uint32_t unit[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { step[k] = dp->step[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * kEntry; }
-    const float bias = dp->bias;
-    const float exact_above = dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY;   // deviations the tables may serve
+    for (int k = 0; k < 8; ++k) { step[k] = F32T ? 0.0f : dp->step[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * kEntry; }
+    const float bias = F32T ? 0.0f : dp->bias;
+    const float exact_above = F32T ? INFINITY : (dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY);   // deviations the tables may serve
     __syncthreads();
 
     const int64_t rows = n * 4;
@@ -152,31 +165,50 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
                 }
             }
         }
-        // two channels per packed float32x2 accumulator, started at the affine offset
-        float2 acc[CH / 2];
-#pragma unroll
-        for (int i = 0; i < CH / 2; ++i) acc[i] = make_float2(bias, bias);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
-            const float2 sk = make_float2(step[k], step[k]);
-            uint32_t e[CH / 2];
-            if (CH == 8) {
-                const uint4 t = *reinterpret_cast<const uint4 *>(table + j * kLine + unit[k]);
-                e[0] = t.x; e[1] = t.y; e[CH / 2 - 2] = t.z; e[CH / 2 - 1] = t.w;
-            } else {
-                const uint2 t = *reinterpret_cast<const uint2 *>(table + j * kLine + unit[k]);
-                e[0] = t.x; e[1] = t.y;
-            }
-#pragma unroll
-            for (int i = 0; i < CH / 2; ++i)
-                acc[i] = fma2(make_float2(level_to_float<0>(e[i]), level_to_float<1>(e[i])), sk, acc[i]);
-        }
         const float sd = live ? __half2float(__ushort_as_half(std16[v])) : 0.0f;
         float o8[CH];
+        if (F32T) {
+            float acc[CH];
 #pragma unroll
-        for (int i = 0; i < CH / 2; ++i) { o8[2 * i] = acc[i].x * sd; o8[2 * i + 1] = acc[i].y * sd; }
-        if (fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
+            for (int i = 0; i < CH; ++i) acc[i] = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
+                if (CH == 4) {
+                    const float4 t = *reinterpret_cast<const float4 *>(table + j * kLine + unit[k]);
+                    acc[0] += t.x; acc[1] += t.y; acc[CH - 2] += t.z; acc[CH - 1] += t.w;
+                } else {
+                    const float2 t = *reinterpret_cast<const float2 *>(table + j * kLine + unit[k]);
+                    acc[0] += t.x; acc[1] += t.y;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < CH; ++i) o8[i] = acc[i] * sd;
+        } else {
+            // two channels per packed float32x2 accumulator, started at the affine offset
+            float2 acc[CH / 2];
+#pragma unroll
+            for (int i = 0; i < CH / 2; ++i) acc[i] = make_float2(bias, bias);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
+                const float2 sk = make_float2(step[k], step[k]);
+                uint32_t e[CH / 2];
+                if (CH == 8) {
+                    const uint4 t = *reinterpret_cast<const uint4 *>(table + j * kLine + unit[k]);
+                    e[0] = t.x; e[1] = t.y; e[CH / 2 - 2] = t.z; e[CH / 2 - 1] = t.w;
+                } else {
+                    const uint2 t = *reinterpret_cast<const uint2 *>(table + j * kLine + unit[k]);
+                    e[0] = t.x; e[1] = t.y;
+                }
+#pragma unroll
+                for (int i = 0; i < CH / 2; ++i)
+                    acc[i] = fma2(make_float2(level_to_float<0>(e[i]), level_to_float<1>(e[i])), sk, acc[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < CH / 2; ++i) { o8[2 * i] = acc[i].x * sd; o8[2 * i + 1] = acc[i].y * sd; }
+        }
+        if (!F32T && fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
             // too coarse for this deviation: the float32 codewords themselves, summed in stage order
             float ex[CH];
 #pragma unroll
@@ -265,6 +297,36 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
     if (bad && st && slice == 0) atomicAdd(&st->bad_codes, bad);   // every slice sees the same codes
 }
 
+// True when more than an eighth of a sample of up to 256 deviations is beyond the level tables' reach.
+// Uniform over the CTA (and over all CTAs of a launch: they read the same sample).
+__device__ __forceinline__ bool sample_wants_float32(const uint16_t *__restrict__ std16, int64_t n,
+                                                  const uint8_t *__restrict__ dsec)
+{
+    const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
+    const float exact_above = dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY;
+    const int64_t samples = n < 256 ? n : 256, every = n < 256 ? 1 : n >> 8;
+    const bool beyond = threadIdx.x < samples &&
+                        fabsf(__half2float(__ushort_as_half(std16[threadIdx.x * every]))) > exact_above;
+    const int far = __syncthreads_count(beyond);
+    return (int64_t)far * 8 > samples;
+}
+
+// PICK: with up to 1536 codes per stage and 16-bit outputs both kinds of table fit, and which one
+// is faster depends on the deviations: level tables (8-channel slices) while most rows are within
+// their reach, float32 tables (4-channel slices) when many rows would take the exact route.  Both
+// kernels are launched; every CTA of both looks at the same sample of up to 256 deviations, so they
+// agree, and the kernel that is not wanted (PICK 1: levels, PICK 2: float32) returns at once.
+template <int DT, int CH, bool F32T, int PICK>
+__global__ void __launch_bounds__(kDecThreads, 1)
+decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                     const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
+                     int64_t stride, rvq_status *st)
+{
+    extern __shared__ __align__(128) uint8_t table[];
+    if (PICK != 0 && sample_wants_float32(std16, n, dsec) != (PICK == 2)) return;
+    decode_sliced_body<DT, CH, F32T>(s, codes, std16, n, dsec, cb, out, stride, st, table);
+}
+
 }  // namespace
 
 int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
@@ -278,30 +340,38 @@ int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std1
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return RVQ_ERR_DEVICE;
-    const int ch = decode_slice_channels(s.K), ns = 32 / ch;
-    const size_t smem = (size_t)s.K * 16 * ch;
+    // which tables: see prepared.cuh
+    const bool both = decode_levels_supported(s) && s.K <= kDecodeWideK;      // decided on the device
     const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
-    int parts = sms / ns;
-    if (parts > tiles) parts = (int)tiles;
-    if (parts < 1) parts = 1;
-    auto launch = [&](auto kernel) -> int {
+    auto launch = [&](auto kernel, int ch, bool f32t) -> int {
+        const int ns = 32 / ch;
+        const size_t smem = (size_t)s.K * (f32t ? 32 : 16) * ch;
+        int parts = sms / ns;
+        if (parts > tiles) parts = (int)tiles;
+        if (parts < 1) parts = 1;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return RVQ_ERR_LAUNCH;
         kernel<<<parts * ns, kDecThreads, smem, stream>>>(s, codes, std16, n, p + off, cb, out, stride, st);
         return check_launch();
     };
-    if (ch == 8) {
+    if (both) {
+        int rc;
+        if (s.dtype == RVQ_BF16) {
+            if ((rc = launch(decode_sliced_kernel<RVQ_BF16, 8, false, 1>, 8, false)) != RVQ_OK) return rc;
+            return launch(decode_sliced_kernel<RVQ_BF16, 4, true, 2>, 4, true);
+        }
+        if ((rc = launch(decode_sliced_kernel<RVQ_F16, 8, false, 1>, 8, false)) != RVQ_OK) return rc;
+        return launch(decode_sliced_kernel<RVQ_F16, 4, true, 2>, 4, true);
+    }
+    if (decode_exact_tables(s)) {
         switch (s.dtype) {
-        case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32, 8>);
-        case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16, 8>);
-        default: return launch(decode_sliced_kernel<RVQ_F16, 8>);
+        case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32, 4, true, 0>, 4, true);
+        case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16, 4, true, 0>, 4, true);
+        default: return launch(decode_sliced_kernel<RVQ_F16, 4, true, 0>, 4, true);
         }
     }
-    switch (s.dtype) {
-    case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32, 4>);
-    case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16, 4>);
-    default: return launch(decode_sliced_kernel<RVQ_F16, 4>);
-    }
+    if (s.dtype == RVQ_BF16) return launch(decode_sliced_kernel<RVQ_BF16, 4, false, 0>, 4, false);
+    return launch(decode_sliced_kernel<RVQ_F16, 4, false, 0>, 4, false);
 }
 
 }  // namespace rvq

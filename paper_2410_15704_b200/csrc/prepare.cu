@@ -32,7 +32,7 @@ static size_t decode_section_offset(const Shape &s)
 size_t prepared_bytes(const Shape &s)
 {
     size_t b = decode_section_offset(s);
-    if (decode_sliced_supported(s)) b += 256 + decode_table_bytes(s.K);
+    if (decode_levels_prepared(s)) b += 256 + decode_table_bytes(s.K);
     return (b + 255) / 256 * 256;
 }
 
@@ -140,7 +140,7 @@ prepare_params_kernel(Shape s, const StagePartial *__restrict__ part, PreparedHe
     if (r == 0) {
         hdr->magic = kPreparedMagic; hdr->R = s.R; hdr->K = s.K; hdr->gd = s.gd;
         hdr->slots = slots_per_stage(s.K);
-        hdr->decode_offset = decode_sliced_supported(s)
+        hdr->decode_offset = decode_levels_prepared(s)
             ? (uint32_t)((kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256) : 0u;
         if (dp) {
             float b = 0.0f, e = 0.0f;
@@ -231,7 +231,7 @@ int launch_prepare(const Shape &s, const float *cb, void *prepared, cudaStream_t
     StageParams *sp = reinterpret_cast<StageParams *>(p + kPreparedParamsOffset);
     StageMaxima *mx = reinterpret_cast<StageMaxima *>(p + kPreparedMaximaOffset);
     StagePartial *part = reinterpret_cast<StagePartial *>(p + kPreparedPartialsOffset);
-    const bool dec = decode_sliced_supported(s);
+    const bool dec = decode_levels_prepared(s);
     const size_t off = decode_section_offset(s);
     DecodeParams *dp = dec ? reinterpret_cast<DecodeParams *>(p + off) : nullptr;
     float *lo = dec ? reinterpret_cast<float *>(p + off + 128) : nullptr;   // per-stage minima, second half of the parameter block

@@ -21,6 +21,12 @@ Parity status of each function against something other than itself
                         the population (ddof=0) standard deviation are this
                         oracle's reading of a paper that states neither:
                         parity unpinned for those two choices.
+  lloyd / kmeans_init   pinned: scipy's kmeans2 from the same start, closed-form
+                        cluster means, empty-cluster and zero-iteration cases,
+                        and the C encoder reproducing the assignments; WHICH
+                        k-means the paper runs (start, iteration count, empty
+                        clusters) is not stated: parity unpinned for those.
+  learn_step            encode followed by ema_update (both pinned above)
 """
 from __future__ import annotations
 
@@ -170,6 +176,76 @@ def ema_update(x, codes, codebooks, ema_count, ema_sum, decay, eps, layout=CONTI
     cnt, sm = ema_stats(x, codes, codebooks, layout, ddof)
     n2, m2, cb = ema_normalise(cnt, sm, ema_count, ema_sum, decay, eps)
     return dict(count=cnt, sum=sm, ema_count=n2, ema_sum=m2, codebooks=cb)
+
+
+def learn_step(x, codebooks, ema_count, ema_sum, decay, eps, group_dim=32, layout=CONTIGUOUS, ddof=0):
+    """One codebook-learning step (Section 3): the batch is encoded with the
+    current codebooks and these assignments feed the EMA update."""
+    enc = encode(x, codebooks, group_dim, layout, ddof)
+    out = ema_update(x, enc["codes"], codebooks, ema_count, ema_sum, decay, eps, layout, ddof)
+    out["codes"], out["std_bits"] = enc["codes"], enc["std_bits"]
+    return out
+
+
+def scaled_groups(x, group_dim=32, layout=CONTIGUOUS, ddof=0):
+    """Section 2.2 / 3.1: every head vector divided by its standard deviation,
+    then cut into groups; returns the group rows [n * G][group_dim] (row v*G+g).
+    A vector without a usable deviation gives zero rows."""
+    x = _f64(x)
+    n, d = x.shape
+    G = d // group_dim
+    mu = x.sum(axis=1, keepdims=True) / d
+    s = np.sqrt(((x - mu) ** 2).sum(axis=1, keepdims=True) / (d - ddof))
+    ok = np.isfinite(s) & (s > 0)
+    z = np.where(ok, x / np.where(ok, s, 1.0), 0.0)
+    if layout == CONTIGUOUS:                      # element i of group g is channel g*gd + i
+        zg = z.reshape(n, G, group_dim)
+    else:                                         # ... or channel i*G + g
+        zg = z.reshape(n, group_dim, G).transpose(0, 2, 1)
+    return np.ascontiguousarray(zg).reshape(n * G, group_dim)
+
+
+def nearest(z, c, block=512):
+    """Index of the nearest row of ``c`` (squared Euclidean distance, direct
+    form, lowest index on ties) for every row of ``z``."""
+    z, c = _f64(z), _f64(c)
+    out = np.empty(len(z), np.int64)
+    for lo in range(0, len(z), block):
+        d = ((z[lo:lo + block, None, :] - c[None, :, :]) ** 2).sum(axis=2)
+        out[lo:lo + block] = d.argmin(axis=1)
+    return out
+
+
+def lloyd(z, c0, iters):
+    """``iters`` iterations of Lloyd's k-means on the rows of ``z`` from the
+    centroids ``c0``: assign every row to its nearest centroid, move every
+    centroid to the mean of its rows; a centroid without rows stays."""
+    z, c = _f64(z), _f64(c0).copy()
+    K = len(c)
+    for _ in range(iters):
+        a = nearest(z, c)
+        cnt = np.bincount(a, minlength=K)
+        sm = np.zeros_like(c)
+        np.add.at(sm, a, z)
+        filled = cnt > 0
+        c[filled] = sm[filled] / cnt[filled, None]
+    return c
+
+
+def kmeans_init(x, seed_rows, iters, group_dim=32, layout=CONTIGUOUS, ddof=0):
+    """Codebook initialisation (Section 3: every codebook starts from k-means):
+    stage r runs Lloyd's iterations on the stage-r inputs of the batch (the
+    scaled group rows minus the chosen codewords of the earlier stages), from
+    the centroids ``z_r[seed_rows[r]]``.  ``seed_rows`` is int [R][K] with group
+    row numbers v*G+g.  Returns float64 codebooks [R][K][group_dim]."""
+    z = scaled_groups(x, group_dim, layout, ddof)
+    seed_rows = np.asarray(seed_rows, dtype=np.int64)
+    cbs = []
+    for r in range(seed_rows.shape[0]):
+        c = lloyd(z, z[seed_rows[r]], iters)
+        z = z - c[nearest(z, c)]
+        cbs.append(c)
+    return np.stack(cbs)
 
 
 def code_bits(K: int) -> int:

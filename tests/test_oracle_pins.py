@@ -386,6 +386,93 @@ def test_ema_special_cases_and_invariants():
 
 # ---------------------------------------------------------------- generators
 
+# ---------------------------------------------------------------- k-means initialisation (Section 3)
+
+def blobs(seed=11, K=12, per=40, gd=32, spread=0.05):
+    g = np.random.default_rng(seed)
+    centres = g.normal(size=(K, gd)) * 3.0
+    labels = np.repeat(np.arange(K), per)
+    z = centres[labels] + spread * g.normal(size=(K * per, gd))
+    perm = g.permutation(len(z))
+    return z[perm], labels[perm], centres
+
+
+def test_lloyd_matches_scipy_kmeans2():
+    from scipy.cluster.vq import kmeans2
+    g = np.random.default_rng(5)
+    z = g.normal(size=(3000, 32)) * g.uniform(0.2, 3.0, size=(1, 32))
+    c0 = z[g.choice(len(z), 48, replace=False)]
+    for iters in (1, 4, 9):
+        ref, _ = kmeans2(z, c0.copy(), iter=iters, minit="matrix")
+        np.testing.assert_allclose(oracle.lloyd(z, c0, iters), ref, rtol=0, atol=1e-12)
+
+
+def test_lloyd_closed_form_on_separated_clusters():
+    z, labels, _ = blobs()
+    K = labels.max() + 1
+    seeds = np.array([np.flatnonzero(labels == k)[0] for k in range(K)])
+    c = oracle.lloyd(z, z[seeds], 1)
+    means = np.stack([z[labels == k].mean(axis=0) for k in range(K)])
+    np.testing.assert_allclose(c, means, atol=1e-13)
+    np.testing.assert_array_equal(oracle.nearest(z, c), labels)
+    np.testing.assert_allclose(oracle.lloyd(z, z[seeds], 7), means, atol=1e-13)     # a fixed point
+
+
+def test_lloyd_zero_iterations_empty_clusters_and_descent():
+    g = np.random.default_rng(9)
+    z = g.normal(size=(500, 8))
+    c0 = z[[3, 3, 17, 400]] .copy()                  # centroid 1 duplicates centroid 0: ties go to 0
+    np.testing.assert_array_equal(oracle.lloyd(z, c0, 0), c0)
+    c = oracle.lloyd(z, c0, 1)
+    np.testing.assert_array_equal(c[1], c0[1])      # had no row in that iteration: stays where it was
+    assert not np.array_equal(c[0], c0[0])
+    cost = []
+    for t in range(6):
+        ct = oracle.lloyd(z, c0, t)
+        cost.append(((z - ct[oracle.nearest(z, ct)]) ** 2).sum())
+    assert all(b <= a + 1e-9 for a, b in zip(cost, cost[1:]))
+
+
+@pytest.mark.parametrize("layout", [oracle.CONTIGUOUS, oracle.STRIDED])
+def test_kmeans_init_stages_agree_with_the_encoder(layout):
+    """The numpy k-means path and the C encoder are separate code: the encoder, given the
+    codebooks k-means produced, must find the same assignments and leave the same residual."""
+    g = np.random.default_rng(21)
+    n, R, K = 96, 3, 16
+    x = g.normal(size=(n, 128)) * g.uniform(0.3, 3.0, size=(1, 128))
+    seeds = np.stack([g.choice(n * 4, K, replace=False) for _ in range(R)])
+    cbs = oracle.kmeans_init(x, seeds, 4, 32, layout)
+    assert cbs.shape == (R, K, 32)
+    # zero iterations: stage 0 is the scaled rows themselves
+    z = oracle.scaled_groups(x, 32, layout)
+    np.testing.assert_array_equal(oracle.kmeans_init(x, seeds, 0, 32, layout)[0], z[seeds[0]])
+    enc = oracle.encode(x, cbs, 32, layout, want_residual=True)
+    zr = z.copy()
+    for r in range(R):
+        a = oracle.nearest(zr, cbs[r])
+        np.testing.assert_array_equal(enc["codes"][:, :, r].reshape(-1), a)
+        zr = zr - cbs[r][a]
+    np.testing.assert_allclose(enc["residual"].reshape(-1, 32), zr, atol=1e-12)
+    # every stage lowers the residual energy, and more iterations do not raise it
+    e4 = (zr ** 2).sum()
+    assert e4 < (z ** 2).sum()
+    enc0 = oracle.encode(x, oracle.kmeans_init(x, seeds, 0, 32, layout), 32, layout, want_residual=True)
+    assert e4 < (enc0["residual"] ** 2).sum()
+
+
+def test_learn_step_is_encode_then_update():
+    x, cb = small_problem(seed=8, n=200, R=3, K=16)
+    N0, M0 = np.ones(cb.shape[:2]), cb.astype(np.float64).copy()
+    out = oracle.learn_step(x, cb, N0, M0, 0.0, 0.0)
+    # decay 0, no smoothing: every used codeword moves to the mean of the stage inputs it was given
+    z = oracle.scaled_groups(x)
+    for r in range(cb.shape[0]):
+        a = out["codes"][:, :, r].reshape(-1)
+        for j in np.unique(a):
+            np.testing.assert_allclose(out["codebooks"][r, j], z[a == j].mean(axis=0), atol=1e-12)
+        z = z - cb[r][a]
+
+
 def test_generators_are_seeded_and_shaped():
     a = rvq_synth.tiny(64)
     b = rvq_synth.tiny(64)

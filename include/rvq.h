@@ -164,12 +164,15 @@ int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n,
 /*
  * Decode (Section 2.2, last sentence; Section 3.2).  For every head vector and
  * channel c = channel(g, i): x_out[c] = std * sum_r C_r[code[g][r]][i], summed
- * in float32 and rounded once to x_dtype.  For 16-bit outputs of dim 128 = 4
- * groups of 32 with depth <= 8 the codebook entries are read from the prepared
- * block as 15-bit levels of each stage's value range, so the sum before the
- * multiplication by std is within sum_r (max C_r - min C_r) * 2^-16 of the
- * float32 one (the prepared block must then have been built with the same
- * x_dtype); float32 outputs and other shapes gather the float32 codebooks.
+ * in float32 and rounded once to x_dtype.  For dim 128 = 4 groups of 32 with
+ * depth <= 8 the codebook entries are read from shared-memory tables: float32
+ * copies (up to 1792 codes per stage) or, for 16-bit outputs and up to 3072
+ * codes, 15-bit levels of each stage's value range kept in the prepared block.
+ * With the levels the sum before the multiplication by std is within
+ * err = sum_r (max C_r - min C_r) * 2^-16 of the float32 one; a head vector whose
+ * std would make std * err exceed 0.9e-3 gets the float32 sum instead, so the
+ * value before the final rounding is always within 1e-3 of the exact one.  Other
+ * shapes gather the float32 codebooks from global memory.
  *   codes, std_f16  in   as produced by rvq_encode
  *   x_out           out  n rows of x_dtype, row v at element v * out_row_stride
  * A code >= K is read as code 0 and counted in status->bad_codes.
@@ -222,6 +225,50 @@ int rvq_ema_stats(const rvq_config *cfg /* host */, const void *x, int64_t n, in
 int rvq_ema_apply(const rvq_config *cfg /* host */, const float *batch_count,
                   const float *batch_sum, float *codebooks, float *ema_count, float *ema_sum,
                   float decay, float eps, void *stream /* cudaStream_t */);
+
+/*
+ * One codebook-learning step (Section 3: the codebooks follow the encoder's own
+ * assignments by exponential moving average, batch after batch): the batch is
+ * encoded with the current codebooks, the statistics of these assignments update
+ * N, M and the codebooks as under rvq_ema_update, and the prepared block is
+ * rebuilt for the new codebooks.  Same results as rvq_encode_stats, rvq_ema_apply
+ * and rvq_prepare_codebooks called in turn.
+ *   codebooks, prepared   in/out
+ *   ema_count, ema_sum    in/out  N [R][K] and M [R][K][group_dim]
+ *   codes, std_f16        out     the batch encoded with the codebooks as they came in
+ *   workspace                     rvq_workspace_bytes(cfg, n) bytes, 256-byte aligned
+ */
+int rvq_learn_step(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
+                   float *codebooks, void *prepared, float *ema_count, float *ema_sum, void *codes,
+                   uint16_t *std_f16, float decay, float eps, void *workspace, size_t workspace_bytes,
+                   rvq_status *status, void *stream /* cudaStream_t */);
+
+/*
+ * k-means initialisation of the codebooks on one batch (Section 3: "we
+ * initialize each codebook using k-means"; the paper gives no further detail,
+ * so the variant is this library's: plain Lloyd iterations).  Stage r works on
+ * the stage-r inputs of the batch -- the scaled group rows minus the centroids
+ * chosen at the earlier stages -- starting from the rows seed_rows[r][0..K) of
+ * that input: `iterations` times every row is assigned to its nearest centroid
+ * (exact squared distance, lowest index on ties) and every centroid moves to the
+ * mean of its rows; a centroid without rows stays where it is.
+ *   seed_rows   in   device, int64 [R][K]: group row numbers v * G + g in
+ *                    [0, n * G), drawn by the caller (the library draws no
+ *                    random numbers); a number out of range reads row 0
+ *   iterations  in   0..1000 (0: the codebooks are the seed rows)
+ *   codebooks   out  float32 [R][K][group_dim]
+ *   prepared    out  ready for rvq_encode / rvq_decode with these codebooks
+ *   workspace        rvq_kmeans_workspace_bytes(cfg, n) bytes, 256-byte aligned:
+ *                    the float32 stage inputs (n * dim * 4 bytes) and the
+ *                    per-stage scratch
+ * group_dim 32 with a power-of-two number of groups only
+ * (RVQ_ERR_UNSUPPORTED otherwise).
+ */
+size_t rvq_kmeans_workspace_bytes(const rvq_config *cfg /* host */, int64_t n);
+int rvq_kmeans_init(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
+                    const int64_t *seed_rows, int32_t iterations, float *codebooks, void *prepared,
+                    void *workspace, size_t workspace_bytes, rvq_status *status,
+                    void *stream /* cudaStream_t */);
 
 /*
  * rvq_ema_update without a workspace argument.  (The paper has no counterpart;

@@ -74,12 +74,19 @@ def _load() -> ctypes.CDLL:
     lib.rvq_ema_update_static.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, ctypes.c_float,
                                           ctypes.c_float, vp, vp]
     lib.rvq_ema_static_scratch_bytes.restype = sz
+    lib.rvq_learn_step.restype = ctypes.c_int
+    lib.rvq_learn_step.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
+                                   vp, sz, vp, vp]
+    lib.rvq_kmeans_workspace_bytes.restype = sz
+    lib.rvq_kmeans_workspace_bytes.argtypes = [cfgp, i64]
+    lib.rvq_kmeans_init.restype = ctypes.c_int
+    lib.rvq_kmeans_init.argtypes = [cfgp, vp, i64, i64, vp, ctypes.c_int32, vp, vp, vp, sz, vp, vp]
     return lib
 
 
 lib = _load()
 
-EXPORTS = ("rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
+EXPORTS = ("rvq_learn_step", "rvq_kmeans_workspace_bytes", "rvq_kmeans_init", "rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
            "rvq_prepare_codebooks", "rvq_workspace_bytes", "rvq_encode", "rvq_decode",
            "rvq_ema_update")
 
@@ -212,6 +219,32 @@ def rvq_ema_update_static(cfg, x, n, x_row_stride, codes, codebooks, ema_count, 
                                    _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_ema_update_static")
+    return rc
+
+
+def rvq_learn_step(cfg, x, n, x_row_stride, codebooks, prepared, ema_count, ema_sum, codes, std_f16,
+                   decay, eps, workspace, workspace_bytes, status=None, stream=None, check=True) -> int:
+    """Encode the batch, update N, M and the codebooks from its assignments, rebuild the prepared block."""
+    rc = lib.rvq_learn_step(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
+                            _ptr(ema_count), _ptr(ema_sum), _ptr(codes), _ptr(std_f16), decay, eps,
+                            _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_learn_step")
+    return rc
+
+
+def rvq_kmeans_workspace_bytes(cfg: rvq_config, n: int) -> int:
+    return int(lib.rvq_kmeans_workspace_bytes(ctypes.byref(cfg), n))
+
+
+def rvq_kmeans_init(cfg, x, n, x_row_stride, seed_rows, iterations, codebooks, prepared, workspace,
+                    workspace_bytes, status=None, stream=None, check=True) -> int:
+    """Stage-wise k-means initialisation of the codebooks from the int64 [R][K] seed rows."""
+    rc = lib.rvq_kmeans_init(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(seed_rows), iterations,
+                             _ptr(codebooks), _ptr(prepared), _ptr(workspace), workspace_bytes,
+                             _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_kmeans_init")
     return rc
 
 

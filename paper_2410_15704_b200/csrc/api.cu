@@ -35,6 +35,7 @@ int make_shape(const rvq_config *c, Shape *s)
     s->per_vector = s->G * s->R;
     s->code_bytes = (s->per_vector * s->bits + 31) / 32 * 4;
     s->elem_bytes = c->x_dtype == RVQ_F32 ? 4 : 2;
+    s->raw = 0;
     return RVQ_OK;
 }
 
@@ -240,6 +241,54 @@ int rvq_ema_update(const rvq_config *cfg, const void *x, int64_t n, int64_t x_ro
                         (cudaStream_t)stream) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
     return launch_ema_apply(s, bc, bs, codebooks, ema_count, ema_sum, decay, eps, (cudaStream_t)stream);
+}
+
+int rvq_learn_step(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                   float *codebooks, void *prepared, float *ema_count, float *ema_sum, void *codes,
+                   uint16_t *std_f16, float decay, float eps, void *workspace, size_t workspace_bytes,
+                   rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if (!ema_count || !ema_sum || !workspace || !codebooks || !prepared) return RVQ_ERR_BADARG;
+    if (!(decay >= 0.0f && decay <= 1.0f) || !(eps >= 0.0f)) return RVQ_ERR_BADARG;
+    if (!aligned16(ema_sum) || !aligned256(workspace)) return RVQ_ERR_ALIGN;
+    if (workspace_bytes < ema_workspace_bytes(s)) return RVQ_ERR_WORKSPACE;
+    // same carving as rvq_ema_update: counts | batch counts | batch sums
+    uint8_t *ws = reinterpret_cast<uint8_t *>(workspace);
+    float *bc = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s));
+    float *bs = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s) +
+                                          ((size_t)s.R * s.K * sizeof(float) + 255) / 256 * 256);
+    rc = rvq_encode_stats(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, bc, bs, workspace,
+                          workspace_bytes, status, stream);
+    if (rc != RVQ_OK) return rc;
+    rc = launch_ema_apply(s, bc, bs, codebooks, ema_count, ema_sum, decay, eps, (cudaStream_t)stream);
+    if (rc != RVQ_OK) return rc;
+    return launch_prepare(s, codebooks, prepared, (cudaStream_t)stream);
+}
+
+size_t rvq_kmeans_workspace_bytes(const rvq_config *cfg, int64_t n)
+{
+    Shape s;
+    return make_shape(cfg, &s) == RVQ_OK ? kmeans_workspace_bytes(s, n) : 0;
+}
+
+int rvq_kmeans_init(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                    const int64_t *seed_rows, int32_t iterations, float *codebooks, void *prepared,
+                    void *workspace, size_t workspace_bytes, rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if (!encode_tensor_supported(s)) return RVQ_ERR_UNSUPPORTED;
+    if ((rc = check_rows(s, x, n, x_row_stride)) != RVQ_OK) return rc;
+    if (n < 1 || !seed_rows || !codebooks || !prepared || !workspace) return RVQ_ERR_BADARG;
+    if (iterations < 0 || iterations > 1000) return RVQ_ERR_BADARG;
+    if (!aligned16(codebooks) || !aligned256(prepared) || !aligned256(workspace)) return RVQ_ERR_ALIGN;
+    if (workspace_bytes < kmeans_workspace_bytes(s, n)) return RVQ_ERR_WORKSPACE;
+    return launch_kmeans(s, x, n, x_row_stride, seed_rows, iterations, codebooks, prepared, workspace, status,
+                         (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -17,6 +17,7 @@ struct Shape {
     int per_vector;       // G * R codes per head vector
     int code_bytes;       // bytes of one head vector's codes
     int elem_bytes;       // bytes of one x element
+    int raw;              // library-internal: the rows are stage inputs already (no deviation, no scaling)
 };
 
 // Fills `s` from a caller config; returns RVQ_OK or the error to hand back.
@@ -46,6 +47,10 @@ int launch_ema_apply(const Shape &s, const float *batch_count, const float *batc
                      float *ema_count, float *ema_sum, float decay, float eps, cudaStream_t stream);
 size_t ema_workspace_bytes(const Shape &s);     // all of rvq_ema_update's scratch
 size_t ema_stats_scratch_bytes(const Shape &s); // the part rvq_ema_stats itself needs
+size_t kmeans_workspace_bytes(const Shape &s, int64_t n);
+int launch_kmeans(const Shape &s, const void *x, int64_t n, int64_t stride, const int64_t *seed_rows,
+                  int iterations, float *codebooks, void *prepared, void *workspace, rvq_status *st,
+                  cudaStream_t stream);
 size_t prepared_bytes(const Shape &s);
 int launch_prepare(const Shape &s, const float *cb, void *prepared, cudaStream_t stream);
 

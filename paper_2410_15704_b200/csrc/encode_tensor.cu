@@ -443,10 +443,11 @@ encode_tensor_kernel(const Params p)
                 for (int k = 0; k < G; ++k) ss += __shfl_sync(0xFFFFFFFFu, b, base + k);
                 dev = sqrtf(ss / (float)(s.dim - s.ddof));
             }
-            const bool deg = deviation_is_degenerate(dev) || !valid;
+            // (raw rows are stage inputs already: taken as they are, no deviation stored)
+            const bool deg = s.raw ? !valid : (deviation_is_degenerate(dev) || !valid);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) z[i] = deg ? 0.0f : z[i] / dev;
-            if (valid && g == 0) {
+            for (int i = 0; i < 32; ++i) z[i] = deg ? 0.0f : (s.raw ? z[i] : z[i] / dev);
+            if (valid && g == 0 && !s.raw) {
                 const uint16_t hb = deviation_is_degenerate(dev) ? (uint16_t)0 : __half_as_ushort(__float2half_rn(dev));
                 p.std16[v] = hb;
                 if (deviation_is_degenerate(dev)) ++n_degenerate;

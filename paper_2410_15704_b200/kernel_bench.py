@@ -4,6 +4,8 @@
   python paper_2410_15704_b200/kernel_bench.py encode key_cache:4096 value_cache:32768 tiny:4096
   python paper_2410_15704_b200/kernel_bench.py decode decode_bandwidth:131072
   python paper_2410_15704_b200/kernel_bench.py ema ema_learning:131072
+  python paper_2410_15704_b200/kernel_bench.py learn_step ema_learning:131072
+  python paper_2410_15704_b200/kernel_bench.py kmeans ema_learning:131072 --iterations 10
 
 A case is `<workload>:<tokens>` (workload names of `rvq_synth`; `tiny:<n>` takes a vector count).  Each
 launch is timed with CUDA events on the launching stream after three warm-up launches; before every timed
@@ -69,7 +71,9 @@ def config_of(w, bits=None):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "ema"])
+    ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "ema", "learn_step",
+                                       "kmeans"])
+    ap.add_argument("--iterations", type=int, default=10, help="Lloyd iterations per stage (kmeans)")
     ap.add_argument("cases", nargs="+")
     ap.add_argument("--reps", type=int, default=10)
     args = ap.parse_args()
@@ -118,7 +122,19 @@ def main():
                 x = torch.from_numpy(w.x).to(rvq.TORCH_DTYPE[cfg.x_dtype]).cuda()
                 bc = torch.empty(R, K, device="cuda")
                 bs = torch.empty(R, K, gd, device="cuda")
-                if args.kernel == "encode":
+                if args.kernel == "learn_step":
+                    cb0 = b.codebooks.clone()
+                    ema_n, ema_m = torch.ones(R, K, device="cuda"), b.codebooks.clone()
+                    fn = lambda: rvq.rvq_learn_step(cfg, x, n, w.dim, b.codebooks, b.prepared, ema_n, ema_m, b.codes,
+                                                    b.std, w.decay, w.eps, b.workspace, b.workspace_bytes, b.status)
+                elif args.kernel == "kmeans":
+                    seeds = torch.from_numpy(np.stack([rvq_synth.randint(rvq_synth.stream_seed(w.seed, f"seed rows {r}"),
+                                                                         K, n * G) for r in range(R)])).cuda()
+                    nbytes = rvq.rvq_kmeans_workspace_bytes(cfg, n)
+                    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+                    fn = lambda: rvq.rvq_kmeans_init(cfg, x, n, w.dim, seeds, args.iterations, b.codebooks, b.prepared,
+                                                     ws, nbytes, b.status)
+                elif args.kernel == "encode":
                     fn = lambda: rvq.rvq_encode(cfg, x, n, w.dim, b.codebooks, b.prepared, b.codes, b.std,
                                                 b.workspace, b.workspace_bytes, b.status)
                 elif args.kernel == "encode_exact":
@@ -132,8 +148,16 @@ def main():
                                    b.workspace, b.workspace_bytes, b.status)
                     fn = lambda: rvq.rvq_ema_stats(cfg, x, n, w.dim, b.codes, b.codebooks, bc, bs,
                                                    b.workspace, b.workspace_bytes, b.status)
-                med, best = timed(fn, args.reps, flush)
-                if args.kernel == "ema":
+                med, best = timed(fn, args.reps if args.kernel != "kmeans" else min(args.reps, 3), flush)
+                if args.kernel == "kmeans":
+                    # assignments made: every iteration of every stage, plus one per stage but the last
+                    sweeps = R * args.iterations + R - 1
+                    flops = 2.0 * gd * K * G * n * sweeps
+                    line.update(ms_median=med, ms_best=best, iterations=args.iterations, assignment_passes=sweeps,
+                                useful_TFLOPs=flops / med / 1e9, frac_tensor=flops / med / 1e9 / tensor,
+                                peak=tensor, peak_source=src, workspace_bytes=nbytes,
+                                wait_timeouts=rvq.read_status(b.status)["wait_timeouts"])
+                elif args.kernel == "ema":
                     nbytes = n * (w.dim * x.element_size() + code_b) + 2 * R * K * (gd + 1) * 4
                     line.update(ms_median=med, ms_best=best, bytes=nbytes, GBps=nbytes / med / 1e6,
                                 frac_hbm=nbytes / med / 1e6 / hbm, peak=hbm, peak_source=src)

@@ -59,5 +59,16 @@ def test_bad_pointers_are_rejected_before_launch():
     assert rvq.lib.rvq_decode(c, 256, 256, 4, 256, 256, 264, 128, None, None) == -2
     assert rvq.lib.rvq_ema_update(c, 256, 4, 128, 256, 256, 256, 256, None, 0.99, 1e-5, 256, 16, None, None) == -4
     assert rvq.lib.rvq_ema_update(c, 256, 4, 128, 256, 256, 256, 256, None, 1.5, 1e-5, 256, 1 << 30, None, None) == -1
+    # learning step and k-means initialisation
+    assert rvq.lib.rvq_learn_step(c, 256, 4, 128, 256, 256, 256, 256, 256, 256, 0.99, 1e-5, 256, 16, None, None) == -4
+    assert rvq.lib.rvq_learn_step(c, 256, 4, 128, 256, 256, None, 256, 256, 256, 0.99, 1e-5, 256, 1 << 30, None, None) == -1
+    big = rvq.rvq_kmeans_workspace_bytes(cfg, 1000)
+    assert big >= 1000 * 128 * 4 and big % 256 == 0
+    assert rvq.lib.rvq_kmeans_init(c, 256, 4, 128, 256, 3, 256, 256, 256, 16, None, None) == -4       # workspace too small
+    assert rvq.lib.rvq_kmeans_init(c, 256, 4, 128, None, 3, 256, 256, 256, 1 << 40, None, None) == -1  # no seed rows
+    assert rvq.lib.rvq_kmeans_init(c, 256, 4, 128, 256, -1, 256, 256, 256, 1 << 40, None, None) == -1
+    odd = rvq.make_config(128, 16, rvq.CONTIGUOUS, 8, 256, 8, rvq.BF16)                                # group_dim 16
+    assert rvq.rvq_kmeans_workspace_bytes(odd, 1000) == 0
+    assert rvq.lib.rvq_kmeans_init(ctypes.byref(odd), 256, 4, 128, 256, 3, 256, 256, 256, 1 << 40, None, None) == -3
     assert rvq.lib.rvq_ema_update(c, 256, 4, 128, 256, None, 256, 256, None, 0.9, 1e-5, 256, 1 << 30, None, None) == -1
     assert rvq.lib.rvq_prepare_codebooks(c, None, 256, None) == -1

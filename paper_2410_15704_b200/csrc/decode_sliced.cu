@@ -9,7 +9,7 @@
 //     16 CH bytes per code = 8 stages x 2 CH bytes.  The 32 / CH slices of a row
 //     tile are handled by as many CTAs; the codes they share come from L2.
 //   - One thread produces the CH channels of one (group row, slice).  It reads
-//     its 8 codes as one 16-byte load (or unpacks them from the bit stream) and
+//     its codes as one 16-byte load (or cuts them out of the packed bit stream) and
 //     visits the stages in an order rotated by its lane, so with CH = 8 the 8
 //     lanes of a quarter warp always touch 8 different 16-byte bank groups
 //     whatever the codes are (with CH = 4 two lanes of a half warp can meet).
@@ -70,6 +70,23 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
 // F32T: the tables hold the float32 codebook entries themselves (16 bytes per stage with
 // CH = 4: the same shared-memory geometry as the 15-bit tables with CH = 8) and the sums are
 // exact float32 sums; otherwise 15-bit levels as described above.
+// Codes r = 0 .. R-1 (R <= 8) of BITS bits each (BITS = 0: `bits`, known at run time only) from the 96-bit
+// window u0:u1:u2, packed two per word into cw[4] (which comes in zeroed).
+template <int BITS, bool FULL = false>      // FULL: R is 8
+__device__ __forceinline__ void cut_codes(uint32_t u0, uint32_t u1, uint32_t u2, int R, uint32_t (&cw)[4], int bits = BITS)
+{
+    const int width = BITS ? BITS : bits;
+    const uint32_t mask = (1u << width) - 1u;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        if (FULL || r < R) {
+            const int o = r * width, k = o >> 5;
+            const uint32_t lo = k == 0 ? u0 : (k == 1 ? u1 : u2), hi = k == 0 ? u1 : (k == 1 ? u2 : 0u);
+            cw[r >> 1] |= (__funnelshift_r(lo, hi, o & 31) & mask) << (16 * (r & 1));
+        }
+    }
+}
+
 template <int DT, int CH, bool F32T>
 __device__ __forceinline__ void
 decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
@@ -119,20 +136,25 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
             if (s.bits == 16 && s.R == 8) {
                 const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + row);
                 cw[0] = c.x; cw[1] = c.y; cw[2] = c.z; cw[3] = c.w;
-            } else if (s.bits == 11 && s.R == 8) {
-                // 88 bits starting at bit 88 g of the vector's 352: a window of up to four words
-                const uint32_t *wv = reinterpret_cast<const uint32_t *>(codes) + v * 11;
-                const int wi = (g * 88) >> 5, sh = (g * 88) & 31;
-                const uint32_t q0 = __ldg(wv + wi), q1 = __ldg(wv + wi + 1), q2 = __ldg(wv + wi + 2);
-                const uint32_t q3 = wi + 3 < 11 ? __ldg(wv + wi + 3) : 0u;
+            } else if (s.R * s.bits <= 96) {
+                // The row's R codes are R * bits <= 96 consecutive bits of the vector's stream, starting
+                // at bit g * R * bits: fetch the (up to four) words that hold them, shift the window
+                // down to bit 0, and cut the codes out of it.
+                const int words = s.code_bytes >> 2;
+                const uint32_t *wv = reinterpret_cast<const uint32_t *>(codes) + v * words;
+                const int bit0 = g * s.R * s.bits, wi = bit0 >> 5, sh = bit0 & 31;
+                const uint32_t q0 = __ldg(wv + wi);
+                const uint32_t q1 = wi + 1 < words ? __ldg(wv + wi + 1) : 0u;
+                const uint32_t q2 = wi + 2 < words ? __ldg(wv + wi + 2) : 0u;
+                const uint32_t q3 = wi + 3 < words ? __ldg(wv + wi + 3) : 0u;
                 const uint32_t u0 = __funnelshift_r(q0, q1, sh), u1 = __funnelshift_r(q1, q2, sh);
                 const uint32_t u2 = __funnelshift_r(q2, q3, sh);
-                // codes at bits 0, 11, ..., 77 of u0:u1:u2
-                const uint32_t c0 = u0 & 0x7FFu, c1 = (u0 >> 11) & 0x7FFu;
-                const uint32_t c2 = __funnelshift_r(u0, u1, 22) & 0x7FFu, c3 = (u1 >> 1) & 0x7FFu;
-                const uint32_t c4 = (u1 >> 12) & 0x7FFu, c5 = __funnelshift_r(u1, u2, 23) & 0x7FFu;
-                const uint32_t c6 = (u2 >> 2) & 0x7FFu, c7 = (u2 >> 13) & 0x7FFu;
-                cw[0] = c0 | (c1 << 16); cw[1] = c2 | (c3 << 16); cw[2] = c4 | (c5 << 16); cw[3] = c6 | (c7 << 16);
+                switch (s.bits) {                  // the usual widths with their offsets known at compile time
+                case 10: if (s.R == 8) cut_codes<10, true>(u0, u1, u2, 8, cw); else cut_codes<10>(u0, u1, u2, s.R, cw); break;
+                case 11: if (s.R == 8) cut_codes<11, true>(u0, u1, u2, 8, cw); else cut_codes<11>(u0, u1, u2, s.R, cw); break;
+                case 12: cut_codes<12>(u0, u1, u2, s.R, cw); break;
+                default: cut_codes<0>(u0, u1, u2, s.R, cw, s.bits); break;
+                }
             } else {
                 const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes;
                 for (int r = 0; r < s.R; ++r)

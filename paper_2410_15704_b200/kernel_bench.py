@@ -6,6 +6,7 @@
   python paper_2410_15704_b200/kernel_bench.py ema ema_learning:131072
   python paper_2410_15704_b200/kernel_bench.py learn_step ema_learning:131072
   python paper_2410_15704_b200/kernel_bench.py kmeans ema_learning:131072 --iterations 10
+  python paper_2410_15704_b200/kernel_bench.py encode ablation:32768 --shape 128,32,6,1024
 
 A case is `<workload>:<tokens>` (workload names of `rvq_synth`; `tiny:<n>` takes a vector count).  Each
 launch is timed with CUDA events on the launching stream after three warm-up launches; before every timed
@@ -74,6 +75,8 @@ def main():
     ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "ema", "learn_step",
                                        "kmeans"])
     ap.add_argument("--iterations", type=int, default=10, help="Lloyd iterations per stage (kmeans)")
+    ap.add_argument("--shape", default=None,
+                    help="dim,group_dim,depth,codes[,layout] of the `ablation` workload, e.g. 128,32,6,1024")
     ap.add_argument("cases", nargs="+")
     ap.add_argument("--reps", type=int, default=10)
     args = ap.parse_args()
@@ -85,12 +88,15 @@ def main():
     for spec in args.cases:
         if args.kernel == "decode" and spec.startswith("decode_bandwidth"):
             runs = [make(spec, layout=0), make(spec, layout=1)]
+        elif spec.startswith("ablation") and args.shape:
+            f = [int(t) for t in args.shape.split(",")]
+            runs = [make(spec, dim=f[0], group_dim=f[1], depth=f[2], size=f[3], layout=f[4] if len(f) > 4 else 0)]
         else:
             runs = [make(spec)]
         for name, w in runs:
             n, G, R, K, gd = w.n, w.groups, w.depth, w.codebook_size, w.group_dim
             code_b = (G * R * w.code_bits + 31) // 32 * 4
-            line = {"kernel": args.kernel, "workload": name, "vectors": n, "K": K, "R": R,
+            line = {"kernel": args.kernel, "workload": name, "vectors": n, "dim": w.dim, "group_dim": gd, "K": K, "R": R,
                     "layout": "strided" if w.layout else "contiguous", "code_bits": w.code_bits}
             if args.kernel == "decode":
                 cfg = config_of(w)

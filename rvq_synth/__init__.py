@@ -244,6 +244,21 @@ def value_cache(tokens: int = 32768, heads: int = 8, seed: int = 1003, size: int
     return w
 
 
+def ablation(tokens: int = 32768, heads: int = 8, dim: int = 128, group_dim: int = 32, depth: int = 8,
+             size: int = 2048, layout: int = CONTIGUOUS, seed: int = 1006) -> Workload:
+    """The codebook-size ablation's shapes (depth 4/6/8, 1024/2048 codes, and
+    other group and head sizes): tokens x heads x dim bf16 Gaussian vectors,
+    Gaussian codebooks shrinking by 0.8 per stage, packed codes, bf16 out."""
+    bits = max(1, int(size - 1).bit_length())
+    w = Workload("ablation", seed, dim, group_dim, layout, depth, size, bits, "bf16", "bf16",
+                 n=tokens * heads, heads=heads)
+    x = normal(stream_seed(seed, "x"), tokens * heads * dim).reshape(tokens * heads, dim)
+    w.x_bits = to_bf16_bits(x)
+    w.x = bf16_bits_to_f32(w.x_bits)
+    w.codebooks = _gaussian_codebooks(seed, depth, size, group_dim, 1.0, 0.8)
+    return w
+
+
 def decode_bandwidth(tokens: int = 131072, heads: int = 8, seed: int = 1004, size: int = 1024,
                      depth: int = 8, layout: int = CONTIGUOUS) -> Workload:
     """Decode-only: uniform uint16 codes, fp16 std = |N(1, 0.25)| + 0.05,
@@ -276,4 +291,5 @@ WORKLOADS = {
     "value_cache": value_cache,
     "decode_bandwidth": decode_bandwidth,
     "ema_learning": ema_learning,
+    "ablation": ablation,
 }

@@ -27,6 +27,11 @@ Parity status of each function against something other than itself
                         k-means the paper runs (start, iteration count, empty
                         clusters) is not stated: parity unpinned for those.
   learn_step            encode followed by ema_update (both pinned above)
+  rope / decode_rope    pinned: the transformers library's Llama rotary helper
+                        (half-split pairing), complex multiplication (adjacent
+                        pairing), identity at position 0, norm preservation,
+                        additivity in the position, the relative-position
+                        property of the inner product
 """
 from __future__ import annotations
 
@@ -176,6 +181,38 @@ def ema_update(x, codes, codebooks, ema_count, ema_sum, decay, eps, layout=CONTI
     cnt, sm = ema_stats(x, codes, codebooks, layout, ddof)
     n2, m2, cb = ema_normalise(cnt, sm, ema_count, ema_sum, decay, eps)
     return dict(count=cnt, sum=sm, ema_count=n2, ema_sum=m2, codebooks=cb)
+
+
+ROPE_HALVES, ROPE_ADJACENT = 0, 1
+
+
+def rope(x, positions, base=10000.0, style=ROPE_HALVES):
+    """Rotary position embedding of the rows of ``x`` [n][d] at integer
+    ``positions`` [n]: pair k of a row is rotated by the angle
+    positions * base**(-2k/d).  Pairs are channels (k, k + d/2)
+    (ROPE_HALVES, the Llama checkpoints' convention) or (2k, 2k + 1)
+    (ROPE_ADJACENT, RoFormer's).  Section 3: keys are quantized before this
+    rotation, so a decoded key gets it afterwards."""
+    x = _f64(x)
+    n, d = x.shape
+    h = d // 2
+    ang = np.asarray(positions, dtype=np.float64)[:, None] * base ** (-2.0 * np.arange(h) / d)[None, :]
+    c, s_ = np.cos(ang), np.sin(ang)
+    out = np.empty_like(x)
+    if style == ROPE_HALVES:
+        a, b = x[:, :h], x[:, h:]
+        out[:, :h], out[:, h:] = a * c - b * s_, b * c + a * s_
+    else:
+        a, b = x[:, 0::2], x[:, 1::2]
+        out[:, 0::2], out[:, 1::2] = a * c - b * s_, b * c + a * s_
+    return out
+
+
+def decode_rope(codes, std_bits, codebooks, positions, base=10000.0, style=ROPE_HALVES, dim=128,
+                layout=CONTIGUOUS, out_dtype=None):
+    """Decode followed by the rotary embedding, rounded once at the end."""
+    out = rope(decode(codes, std_bits, codebooks, dim, layout), positions, base, style)
+    return out if out_dtype is None else round_to(out, out_dtype)
 
 
 def learn_step(x, codebooks, ema_count, ema_sum, decay, eps, group_dim=32, layout=CONTIGUOUS, ddof=0):

@@ -473,6 +473,67 @@ def test_learn_step_is_encode_then_update():
         z = z - cb[r][a]
 
 
+# ---------------------------------------------------------------- rotary embedding after decode
+
+def test_rope_halves_matches_transformers_llama_helper():
+    import torch
+    from transformers.models.llama.modeling_llama import apply_rotary_pos_emb
+    g = np.random.default_rng(2)
+    n, d, base = 37, 128, 500000.0
+    x = g.normal(size=(n, d))
+    pos = g.integers(0, 100000, size=n)
+    inv = 1.0 / (base ** (torch.arange(0, d, 2, dtype=torch.float64) / d))
+    fr = torch.outer(torch.from_numpy(pos).double(), inv)
+    emb = torch.cat([fr, fr], dim=-1)
+    q = torch.from_numpy(x)[None, None]                                   # [batch][head][token][d]
+    qe, _ = apply_rotary_pos_emb(q, q, emb.cos()[None], emb.sin()[None])
+    np.testing.assert_allclose(oracle.rope(x, pos, base, oracle.ROPE_HALVES), qe[0, 0].numpy(), rtol=0, atol=1e-10)   # angles near 1e5 rad: 1e-11 of rounding
+
+
+def test_rope_adjacent_is_complex_multiplication():
+    g = np.random.default_rng(3)
+    n, d, base = 20, 64, 10000.0
+    x = g.normal(size=(n, d))
+    pos = g.integers(0, 5000, size=n)
+    zc = (x[:, 0::2] + 1j * x[:, 1::2]) * np.exp(1j * pos[:, None] * base ** (-2.0 * np.arange(d // 2) / d)[None, :])
+    out = oracle.rope(x, pos, base, oracle.ROPE_ADJACENT)
+    np.testing.assert_allclose(out[:, 0::2], zc.real, atol=1e-12)
+    np.testing.assert_allclose(out[:, 1::2], zc.imag, atol=1e-12)
+
+
+@pytest.mark.parametrize("style", [oracle.ROPE_HALVES, oracle.ROPE_ADJACENT])
+def test_rope_properties(style):
+    g = np.random.default_rng(4)
+    q, k = g.normal(size=(9, 128)), g.normal(size=(9, 128))
+    zero = np.zeros(9, dtype=np.int64)
+    np.testing.assert_array_equal(oracle.rope(q, zero, 10000.0, style), q)                 # position 0: identity
+    p1, p2 = g.integers(0, 3000, size=9), g.integers(0, 3000, size=9)
+    r1 = oracle.rope(q, p1, 10000.0, style)
+    np.testing.assert_allclose((r1 ** 2).sum(axis=1), (q ** 2).sum(axis=1), rtol=1e-13)   # a rotation
+    np.testing.assert_allclose(oracle.rope(r1, p2, 10000.0, style), oracle.rope(q, p1 + p2, 10000.0, style),
+                               atol=1e-9)                                                  # angles add
+    # the inner product of a rotated query and key depends on the distance of their positions only
+    a = (oracle.rope(q, p1 + 17, 10000.0, style) * oracle.rope(k, p1, 10000.0, style)).sum(axis=1)
+    b = (oracle.rope(q, p2 + 17, 10000.0, style) * oracle.rope(k, p2, 10000.0, style)).sum(axis=1)
+    np.testing.assert_allclose(a, b, atol=1e-8)
+    # and the two pairings are the same rotation up to a permutation of the channels
+    perm = np.concatenate([np.arange(0, 128, 2), np.arange(1, 128, 2)])                    # adjacent -> halves
+    np.testing.assert_allclose(oracle.rope(q, p1, 10000.0, oracle.ROPE_ADJACENT)[:, perm],
+                               oracle.rope(q[:, perm], p1, 10000.0, oracle.ROPE_HALVES), atol=1e-12)
+
+
+def test_decode_rope_is_decode_then_rotation():
+    x, cb = small_problem(seed=12, n=40, R=4, K=16)
+    enc = oracle.encode(x, cb)
+    pos = np.arange(40) * 7
+    plain = oracle.decode(enc["codes"], enc["std_bits"], cb)
+    got = oracle.decode_rope(enc["codes"], enc["std_bits"], cb, pos)
+    np.testing.assert_allclose((got ** 2).sum(axis=1), (plain ** 2).sum(axis=1), rtol=1e-12)
+    np.testing.assert_array_equal(oracle.decode_rope(enc["codes"], enc["std_bits"], cb, 0 * pos), plain)
+    bf = oracle.decode_rope(enc["codes"], enc["std_bits"], cb, pos, out_dtype=oracle.BF16)
+    np.testing.assert_array_equal(bf, oracle.round_to(got, oracle.BF16))
+
+
 def test_generators_are_seeded_and_shaped():
     a = rvq_synth.tiny(64)
     b = rvq_synth.tiny(64)

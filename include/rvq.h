@@ -182,6 +182,35 @@ int rvq_decode(const rvq_config *cfg /* host */, const void *codes, const uint16
                int64_t out_row_stride, rvq_status *status, void *stream /* cudaStream_t */);
 
 /*
+ * Decode followed by the rotary position embedding (Section 3: keys are
+ * quantized before the rotation, so a key read back from the cache still needs
+ * it; done here it costs no second pass over the keys).  With x^ the decoded
+ * head vector in float32 (as under rvq_decode, before rounding), p its position
+ * and (c_k, s_k) = cos_sin[p][k] for pair k:
+ *   pairing RVQ_ROPE_HALVES    (a, b) = (x^[k], x^[k + dim/2])   (Llama checkpoints)
+ *   pairing RVQ_ROPE_ADJACENT  (a, b) = (x^[2k], x^[2k + 1])     (RoFormer)
+ *   a' = a c_k - b s_k ,  b' = b c_k + a s_k ,  rounded once to x_dtype.
+ *   position              in  device int32: head vector v sits at position[v / vectors_per_position]
+ *                             (vectors_per_position = number of KV heads for [token][head][dim] rows);
+ *                             values outside [0, positions) are clamped into it
+ *   cos_sin               in  device float32 [positions][dim/2][2], 16-byte aligned, e.g. from
+ *                             rvq_rope_table
+ * dim 128 in 4 groups of 32, depth <= 8 and up to 1792 codes per stage use float32
+ * shared-memory tables (exact float32 sums); other shapes gather from global memory.
+ */
+enum { RVQ_ROPE_HALVES = 0, RVQ_ROPE_ADJACENT = 1 };
+int rvq_decode_rope(const rvq_config *cfg /* host */, const void *codes, const uint16_t *std_f16,
+                    int64_t n, const float *codebooks, const int32_t *position,
+                    int32_t vectors_per_position, const float *cos_sin, int32_t positions,
+                    int32_t pairing, void *x_out, int64_t out_row_stride, rvq_status *status,
+                    void *stream /* cudaStream_t */);
+
+/* cos_sin[p][k] = (cos, sin)(p * base^(-2k/dim)) for p < positions, k < dim/2, evaluated in
+ * double precision and rounded to float32 (the angles reach 1e5 radians at long context). */
+int rvq_rope_table(int32_t dim, double base, int32_t positions, float *cos_sin /* device */,
+                   void *stream /* cudaStream_t */);
+
+/*
  * One EMA codebook update (Section 3: "update them using exponential moving
  * average with a decay factor of 0.99"; Section 2.1: EMA in place of the
  * codebook loss).  With n_r[j] the number of group rows whose stage-r code is j

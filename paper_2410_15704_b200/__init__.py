@@ -74,6 +74,11 @@ def _load() -> ctypes.CDLL:
     lib.rvq_ema_update_static.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, ctypes.c_float,
                                           ctypes.c_float, vp, vp]
     lib.rvq_ema_static_scratch_bytes.restype = sz
+    lib.rvq_rope_table.restype = ctypes.c_int
+    lib.rvq_rope_table.argtypes = [ctypes.c_int32, ctypes.c_double, ctypes.c_int32, vp, vp]
+    lib.rvq_decode_rope.restype = ctypes.c_int
+    lib.rvq_decode_rope.argtypes = [cfgp, vp, vp, i64, vp, vp, ctypes.c_int32, vp, ctypes.c_int32, ctypes.c_int32,
+                                    vp, i64, vp, vp]
     lib.rvq_learn_step.restype = ctypes.c_int
     lib.rvq_learn_step.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
                                    vp, sz, vp, vp]
@@ -86,7 +91,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 
-EXPORTS = ("rvq_learn_step", "rvq_kmeans_workspace_bytes", "rvq_kmeans_init", "rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
+EXPORTS = ("rvq_rope_table", "rvq_decode_rope", "rvq_learn_step", "rvq_kmeans_workspace_bytes", "rvq_kmeans_init", "rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
            "rvq_prepare_codebooks", "rvq_workspace_bytes", "rvq_encode", "rvq_decode",
            "rvq_ema_update")
 
@@ -219,6 +224,28 @@ def rvq_ema_update_static(cfg, x, n, x_row_stride, codes, codebooks, ema_count, 
                                    _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_ema_update_static")
+    return rc
+
+
+ROPE_HALVES, ROPE_ADJACENT = 0, 1
+
+
+def rvq_rope_table(dim, base, positions, cos_sin, stream=None, check=True) -> int:
+    """Fill cos_sin (float32 [positions][dim/2][2]) with the rotary embedding's cosines and sines."""
+    rc = lib.rvq_rope_table(dim, float(base), positions, _ptr(cos_sin), _stream(stream))
+    if check:
+        _check(rc, "rvq_rope_table")
+    return rc
+
+
+def rvq_decode_rope(cfg, codes, std_f16, n, codebooks, position, vectors_per_position, cos_sin, positions,
+                    pairing, x_out, out_row_stride, status=None, stream=None, check=True) -> int:
+    """Decode and rotate: x_out = RoPE(decode(codes)) at the given positions."""
+    rc = lib.rvq_decode_rope(ctypes.byref(cfg), _ptr(codes), _ptr(std_f16), n, _ptr(codebooks), _ptr(position),
+                             vectors_per_position, _ptr(cos_sin), positions, pairing, _ptr(x_out), out_row_stride,
+                             _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_decode_rope")
     return rc
 
 

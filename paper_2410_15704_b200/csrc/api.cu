@@ -179,6 +179,32 @@ int rvq_decode(const rvq_config *cfg, const void *codes, const uint16_t *std_f16
     return launch_decode_gather(s, codes, std_f16, n, codebooks, x_out, out_row_stride, status, (cudaStream_t)stream);
 }
 
+int rvq_rope_table(int32_t dim, double base, int32_t positions, float *cos_sin, void *stream)
+{
+    if (dim < 2 || dim > 1024 || (dim & 1) || !(base > 1.0) || positions < 0 || (positions > 0 && !cos_sin))
+        return RVQ_ERR_BADARG;
+    if (!aligned16(cos_sin)) return RVQ_ERR_ALIGN;
+    return launch_rope_table(dim, base, positions, cos_sin, (cudaStream_t)stream);
+}
+
+int rvq_decode_rope(const rvq_config *cfg, const void *codes, const uint16_t *std_f16, int64_t n,
+                    const float *codebooks, const int32_t *position, int32_t vectors_per_position,
+                    const float *cos_sin, int32_t positions, int32_t pairing, void *x_out,
+                    int64_t out_row_stride, rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if ((rc = check_rows(s, x_out, n, out_row_stride)) != RVQ_OK) return rc;
+    if (!codebooks || (n > 0 && (!codes || !std_f16 || !position || !cos_sin))) return RVQ_ERR_BADARG;
+    if (vectors_per_position < 1 || positions < 1 || (pairing != RVQ_ROPE_HALVES && pairing != RVQ_ROPE_ADJACENT))
+        return RVQ_ERR_BADARG;
+    if (s.dim & 1) return RVQ_ERR_UNSUPPORTED;
+    if (!aligned16(codebooks) || !aligned16(codes) || !aligned16(cos_sin)) return RVQ_ERR_ALIGN;
+    return launch_decode_rope(s, codes, std_f16, n, codebooks, position, vectors_per_position, cos_sin, positions,
+                              pairing, x_out, out_row_stride, status, (cudaStream_t)stream);
+}
+
 static int check_ema_common(const Shape &s, const void *x, int64_t n, int64_t stride, const void *codes,
                             const float *codebooks)
 {

@@ -87,12 +87,34 @@ __device__ __forceinline__ void cut_codes(uint32_t u0, uint32_t u1, uint32_t u2,
     }
 }
 
-template <int DT, int CH, bool F32T>
+struct RopeArgs {
+    const int32_t *position;      // position of head vector v: position[v / per_position]
+    int per_position;
+    const float2 *table;          // (cos, sin) [positions][64]
+    int positions;
+};
+
+// Codeword element held at place i of slice `slice`.
+template <int CH, int ROPE>
+__device__ __forceinline__ int slice_element(int layout, int slice, int i)
+{
+    if (ROPE == 1 && layout == RVQ_GROUP_STRIDED) return 2 * slice + (i & 1) + 16 * (i >> 1);
+    return slice * CH + i;
+}
+
+// ROPE (float32 tables with 4-channel slices only): the rotary embedding is applied to the decoded
+// head vector before it is rounded and stored (1: pairs are channels (k, k + 64), 2: (2k, 2k + 1)).
+// Both channels of a pair are in one thread, or in two lanes of the head vector's four, for every
+// combination but one: strided groups with half-split pairs, where the partner of element i of a
+// group is element i + 16 of the same group.  There a slice is the elements {2 sl, 2 sl + 1,
+// 2 sl + 16, 2 sl + 17} instead of four consecutive ones.
+template <int DT, int CH, bool F32T, int ROPE = 0>
 __device__ __forceinline__ void
 decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
                    const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
-                   int64_t stride, rvq_status *st, uint8_t *table)
+                   int64_t stride, rvq_status *st, uint8_t *table, RopeArgs ra = RopeArgs())
 {
+    static_assert(ROPE == 0 || (F32T && CH == 4), "rotary decode uses float32 tables with 4-channel slices");
     // table: [K][8 stages][kEntry bytes] in shared memory
     constexpr int NS = 32 / CH;                                  // slices
     if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;   // (a grid sized for another slice count)
@@ -105,9 +127,9 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
         for (int t = tid; t < s.K * 8; t += kDecThreads) {
             const int r = t / s.K, j = t - r * s.K;
             float *dst = reinterpret_cast<float *>(table + (size_t)j * kLine + r * kEntry);
-            const float *src = cb + ((size_t)r * s.K + j) * 32 + slice * CH;
+            const float *src = cb + ((size_t)r * s.K + j) * 32;
 #pragma unroll
-            for (int i = 0; i < CH; ++i) dst[i] = r < s.R ? __ldg(src + i) : 0.0f;
+            for (int i = 0; i < CH; ++i) dst[i] = r < s.R ? __ldg(src + slice_element<CH, ROPE>(s.layout, slice, i)) : 0.0f;
         }
     } else {
         const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256) + (size_t)slice * s.K * CH;
@@ -130,6 +152,30 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
         const bool live = row < rows;
         const int64_t v = live ? row >> 2 : 0;
         const int g = (int)(row & 3);
+        // rotary decode: this row's cosines and sines, asked for first so that they arrive during the gather
+        float2 rc[4];
+        if (ROPE != 0) {
+            // (the launcher sends larger problems elsewhere: a 64-bit division here is a subroutine call
+            // that costs the whole loop its register allocation)
+            const uint32_t token = (uint32_t)v / (uint32_t)ra.per_position;
+            int pos = live ? __ldg(ra.position + token) : 0;
+            pos = min(max(pos, 0), ra.positions - 1);
+            const float2 *cs = ra.table + (size_t)pos * 64;
+            if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) {          // pairs 4 (2 slice + i) + g
+                rc[0] = __ldg(cs + slice * 8 + g); rc[1] = __ldg(cs + slice * 8 + 4 + g);
+            } else if (ROPE == 2 && s.layout != RVQ_GROUP_STRIDED) {   // pairs 16 g + 2 slice + i
+                const float4 cc = __ldg(reinterpret_cast<const float4 *>(cs + g * 16 + slice * 2));
+                rc[0] = make_float2(cc.x, cc.y); rc[1] = make_float2(cc.z, cc.w);
+            } else if (ROPE == 1) {                                    // pairs 32 (g & 1) + 4 slice + i
+                const float4 *q = reinterpret_cast<const float4 *>(cs + (g & 1) * 32 + slice * 4);
+                const float4 lo = __ldg(q), hi = __ldg(q + 1);
+                rc[0] = make_float2(lo.x, lo.y); rc[1] = make_float2(lo.z, lo.w);
+                rc[2] = make_float2(hi.x, hi.y); rc[3] = make_float2(hi.z, hi.w);
+            } else {                                                   // pairs 2 (4 slice + i) + g / 2
+#pragma unroll
+                for (int i = 0; i < 4; ++i) rc[i] = __ldg(cs + (slice * 4 + i) * 2 + (g >> 1));
+            }
+        }
         // the 8 codes of this row as 4 words, stage r in half r
         uint32_t cw[4] = {0u, 0u, 0u, 0u};
         if (live) {
@@ -252,6 +298,37 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
             for (int i = 0; i < CH; ++i) o8[i] = ex[i] * sd;
         }
 
+        if (ROPE != 0) {
+            const bool strided = s.layout == RVQ_GROUP_STRIDED;
+            if (ROPE == 1 && strided) {
+                // places 0, 1 are channels 4 e + g of the first half, places 2, 3 their partners 64 further on
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float a = o8[i], b = o8[i + 2];
+                    o8[i] = a * rc[i].x - b * rc[i].y;
+                    o8[i + 2] = b * rc[i].x + a * rc[i].y;
+                }
+            } else if (ROPE == 2 && !strided) {
+                // channels 32 g + 4 slice + i: pairs (0, 1) and (2, 3) are in this thread
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float a = o8[2 * i], b = o8[2 * i + 1];
+                    o8[2 * i] = a * rc[i].x - b * rc[i].y;
+                    o8[2 * i + 1] = b * rc[i].x + a * rc[i].y;
+                }
+            } else {
+                // the partner is the same place of another group: lane g ^ 2 (half-split pairs, contiguous
+                // groups: channels 32 g + e and 32 (g ^ 2) + e) or lane g ^ 1 (adjacent pairs, strided groups:
+                // channels 4 e + g and 4 e + (g ^ 1))
+                const int other = ROPE == 1 ? 2 : 1;
+                const bool first = (g & other) == 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float b = __shfl_xor_sync(0xFFFFFFFFu, o8[i], other);
+                    o8[i] = first ? o8[i] * rc[i].x - b * rc[i].y : o8[i] * rc[i].x + b * rc[i].y;
+                }
+            }
+        }
         if (DT == RVQ_F32) {
             if (s.layout == RVQ_GROUP_CONTIGUOUS) {
                 if (live) {
@@ -261,9 +338,9 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                         o[i] = make_float4(o8[4 * i], o8[4 * i + 1], o8[4 * i + 2], o8[4 * i + 3]);
                 }
             } else if (live) {
-                float *o = reinterpret_cast<float *>(out) + v * stride + slice * CH * 4 + g;
+                float *o = reinterpret_cast<float *>(out) + v * stride + g;
 #pragma unroll
-                for (int i = 0; i < CH; ++i) o[4 * i] = o8[i];        // channel (CH slice + i) * 4 + g
+                for (int i = 0; i < CH; ++i) o[4 * slice_element<CH, ROPE>(s.layout, slice, i)] = o8[i];   // channel 4 element + g
             }
         } else {
             uint32_t w[CH / 2];
@@ -311,7 +388,7 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                 // keep = element L of groups (g & 1) and (g & 1) + 2, got = element L of the other two
                 const uint32_t even = b1 ? got : keep, odd = b1 ? keep : got;   // groups (0, 2) and (1, 3)
                 if (live)
-                    *reinterpret_cast<uint2 *>(o16 + slice * 16 + g * 4) =
+                    *reinterpret_cast<uint2 *>(o16 + 4 * slice_element<CH, ROPE>(s.layout, slice, g)) =
                         make_uint2(__byte_perm(even, odd, 0x5410), __byte_perm(even, odd, 0x7632));
             }
         }
@@ -349,7 +426,117 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
     decode_sliced_body<DT, CH, F32T>(s, codes, std16, n, dsec, cb, out, stride, st, table);
 }
 
+// Decode with the rotary embedding: float32 tables, 4-channel slices (dim 128, up to 1792 codes).
+template <int DT, int ROPE>
+__global__ void __launch_bounds__(kDecThreads, 1)
+decode_rope_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                   const float *__restrict__ cb, void *__restrict__ out, int64_t stride, rvq_status *st, RopeArgs ra)
+{
+    extern __shared__ __align__(128) uint8_t table[];
+    decode_sliced_body<DT, 4, true, ROPE>(s, codes, std16, n, nullptr, cb, out, stride, st, table, ra);
+}
+
+// Any other shape: one thread per (head vector, pair of channels), codeword entries gathered from
+// global memory, float32 sums in stage order, rotation, one rounding.
+__global__ void __launch_bounds__(256)
+decode_rope_gather_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                          const float *__restrict__ cb, void *__restrict__ out, int64_t stride, rvq_status *st,
+                          RopeArgs ra, int style)
+{
+    const int half = s.dim / 2;
+    const int64_t total = n * half;
+    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < total; t += (int64_t)gridDim.x * 256) {
+        const int64_t v = t / half;
+        const int f = (int)(t - v * half);
+        const int c0 = style == 1 ? f : 2 * f, c1 = style == 1 ? f + half : 2 * f + 1;
+        const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes;
+        float val[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c = h ? c1 : c0;
+            const int g = s.layout == RVQ_GROUP_STRIDED ? c % s.G : c / s.gd;
+            const int i = s.layout == RVQ_GROUP_STRIDED ? c / s.G : c % s.gd;
+            float acc = 0.0f;
+            for (int r = 0; r < s.R; ++r) {
+                uint32_t j = read_code(vec, g * s.R + r, s.bits, s.code_bytes);
+                if (j >= (uint32_t)s.K) { j = 0; if (st && i == 0) atomicAdd(&st->bad_codes, 1u); }
+                acc += __ldg(cb + ((size_t)r * s.K + j) * s.gd + i);
+            }
+            val[h] = acc * __half2float(__ushort_as_half(std16[v]));
+        }
+        int pos = ra.position[v / ra.per_position];
+        pos = min(max(pos, 0), ra.positions - 1);
+        const float2 cs = __ldg(ra.table + (size_t)pos * half + f);
+        store_from_float(out, v * stride + c0, s.dtype, val[0] * cs.x - val[1] * cs.y);
+        store_from_float(out, v * stride + c1, s.dtype, val[1] * cs.x + val[0] * cs.y);
+    }
+}
+
+// (cos, sin) of position * base^(-2k/dim), computed in double precision: the angles reach 1e5 radians.
+__global__ void __launch_bounds__(256)
+rope_table_kernel(int dim, double base, int positions, float2 *__restrict__ table)
+{
+    const int half = dim / 2;
+    const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (t >= (int64_t)positions * half) return;
+    const int p = (int)(t / half), k = (int)(t - (int64_t)p * half);
+    const double ang = (double)p * pow(base, -2.0 * (double)k / (double)dim);
+    table[t] = make_float2((float)cos(ang), (float)sin(ang));
+}
+
 }  // namespace
+
+int launch_rope_table(int dim, double base, int positions, float *table, cudaStream_t stream)
+{
+    const int64_t total = (int64_t)positions * (dim / 2);
+    if (total == 0) return RVQ_OK;
+    rope_table_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(dim, base, positions,
+                                                                             reinterpret_cast<float2 *>(table));
+    return check_launch();
+}
+
+int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16, int64_t n, const float *cb,
+                       const int32_t *position, int per_position, const float *table, int positions, int style,
+                       void *out, int64_t stride, rvq_status *st, cudaStream_t stream)
+{
+    if (n == 0) return RVQ_OK;
+    RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions};
+    if (!decode_exact_tables(s) || n > 0x7FFFFFFF) {
+        const int64_t total = n * (s.dim / 2);
+        int64_t blocks = (total + 255) / 256;
+        if (blocks > 148 * 32) blocks = 148 * 32;
+        decode_rope_gather_kernel<<<(unsigned)blocks, 256, 0, stream>>>(s, codes, std16, n, cb, out, stride, st, ra,
+                                                                        style == 0 ? 1 : 2);
+        return check_launch();
+    }
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return RVQ_ERR_DEVICE;
+    const size_t smem = (size_t)s.K * 128;
+    const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
+    int parts = sms / 8;
+    if (parts > tiles) parts = (int)tiles;
+    if (parts < 1) parts = 1;
+    auto launch = [&](auto kernel) -> int {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return RVQ_ERR_LAUNCH;
+        kernel<<<parts * 8, kDecThreads, smem, stream>>>(s, codes, std16, n, cb, out, stride, st, ra);
+        return check_launch();
+    };
+    if (style == 0) {
+        switch (s.dtype) {
+        case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 1>);
+        case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 1>);
+        default: return launch(decode_rope_kernel<RVQ_F16, 1>);
+        }
+    }
+    switch (s.dtype) {
+    case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 2>);
+    case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 2>);
+    default: return launch(decode_rope_kernel<RVQ_F16, 2>);
+    }
+}
 
 int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
                          const float *cb, const void *prepared, void *out, int64_t stride, rvq_status *st,

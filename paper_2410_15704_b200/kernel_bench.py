@@ -3,6 +3,7 @@
 
   python paper_2410_15704_b200/kernel_bench.py encode key_cache:4096 value_cache:32768 tiny:4096
   python paper_2410_15704_b200/kernel_bench.py decode decode_bandwidth:131072
+  python paper_2410_15704_b200/kernel_bench.py decode_rope decode_bandwidth:131072
   python paper_2410_15704_b200/kernel_bench.py ema ema_learning:131072
   python paper_2410_15704_b200/kernel_bench.py learn_step ema_learning:131072
   python paper_2410_15704_b200/kernel_bench.py kmeans ema_learning:131072 --iterations 10
@@ -72,8 +73,8 @@ def config_of(w, bits=None):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "ema", "learn_step",
-                                       "kmeans"])
+    ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "decode_rope", "ema",
+                                       "learn_step", "kmeans"])
     ap.add_argument("--iterations", type=int, default=10, help="Lloyd iterations per stage (kmeans)")
     ap.add_argument("--shape", default=None,
                     help="dim,group_dim,depth,codes[,layout] of the `ablation` workload, e.g. 128,32,6,1024")
@@ -86,7 +87,7 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     for spec in args.cases:
-        if args.kernel == "decode" and spec.startswith("decode_bandwidth"):
+        if args.kernel in ("decode", "decode_rope") and spec.startswith("decode_bandwidth"):
             runs = [make(spec, layout=0), make(spec, layout=1)]
         elif spec.startswith("ablation") and args.shape:
             f = [int(t) for t in args.shape.split(",")]
@@ -98,7 +99,7 @@ def main():
             code_b = (G * R * w.code_bits + 31) // 32 * 4
             line = {"kernel": args.kernel, "workload": name, "vectors": n, "dim": w.dim, "group_dim": gd, "K": K, "R": R,
                     "layout": "strided" if w.layout else "contiguous", "code_bits": w.code_bits}
-            if args.kernel == "decode":
+            if args.kernel in ("decode", "decode_rope"):
                 cfg = config_of(w)
                 b = rvq.alloc_buffers(cfg, n, w.codebooks)
                 tdt = rvq.TORCH_DTYPE[cfg.x_dtype]
@@ -117,9 +118,21 @@ def main():
                         torch.from_numpy(codes.astype(np.uint16).view(np.int16).reshape(-1)))
                     b.std.copy_(torch.from_numpy(std_bits.view(np.int16)))
                 out = torch.empty(n, w.dim, dtype=tdt, device="cuda")
-                med, best = timed(lambda: rvq.rvq_decode(cfg, b.codes, b.std, n, b.codebooks, b.prepared, out,
-                                                         w.dim, b.status), args.reps, flush)
-                nbytes = n * (code_b + 2 + w.dim * out.element_size())
+                if args.kernel == "decode_rope":
+                    # one position per token (all its heads), 128K context, Llama-3's base, half-split pairs
+                    tokens, max_pos = n // w.heads, 131072
+                    table = torch.empty(max_pos, w.dim // 2, 2, device="cuda")
+                    rvq.rvq_rope_table(w.dim, 500000.0, max_pos, table)
+                    pos = (torch.arange(tokens, device="cuda", dtype=torch.int32) % max_pos).contiguous()
+                    med, best = timed(lambda: rvq.rvq_decode_rope(cfg, b.codes, b.std, n, b.codebooks, pos, w.heads,
+                                                                  table, max_pos, rvq.ROPE_HALVES, out, w.dim,
+                                                                  b.status), args.reps, flush)
+                    extra = w.dim // 2 * 8 // w.heads + 4 // w.heads      # a table row and a position per token
+                else:
+                    med, best = timed(lambda: rvq.rvq_decode(cfg, b.codes, b.std, n, b.codebooks, b.prepared, out,
+                                                             w.dim, b.status), args.reps, flush)
+                    extra = 0
+                nbytes = n * (code_b + 2 + w.dim * out.element_size() + extra)
                 line.update(ms_median=med, ms_best=best, bytes=nbytes, GBps=nbytes / med / 1e6,
                             frac_hbm=nbytes / med / 1e6 / hbm, peak=hbm, peak_source=src)
             else:

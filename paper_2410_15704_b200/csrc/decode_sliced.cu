@@ -123,13 +123,29 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
     const int slice = blockIdx.x % NS, part = blockIdx.x / NS, parts = gridDim.x / NS;
     const int tid = threadIdx.x, lane = tid & 31, rot = lane & 7;
     if (F32T) {
-        // entry (code j, stage r) = channels CH slice .. CH slice + CH - 1 of codeword j of stage r
+        // entry (code j, stage r) = CH channels of codeword j of stage r; consecutive threads fill
+        // consecutive entries (stage fastest), so the shared-memory stores do not collide
         for (int t = tid; t < s.K * 8; t += kDecThreads) {
-            const int r = t / s.K, j = t - r * s.K;
-            float *dst = reinterpret_cast<float *>(table + (size_t)j * kLine + r * kEntry);
+            const int r = t & 7, j = t >> 3;
+            float *dst = reinterpret_cast<float *>(table + (size_t)t * kEntry);
             const float *src = cb + ((size_t)r * s.K + j) * 32;
+            float e[CH];
+            if (r >= s.R) {
 #pragma unroll
-            for (int i = 0; i < CH; ++i) dst[i] = r < s.R ? __ldg(src + slice_element<CH, ROPE>(s.layout, slice, i)) : 0.0f;
+                for (int i = 0; i < CH; ++i) e[i] = 0.0f;
+            } else if (CH == 4 && slice_element<CH, ROPE>(s.layout, slice, 1) == slice * CH + 1 &&
+                       slice_element<CH, ROPE>(s.layout, slice, 2) == slice * CH + 2) {
+                const float4 q = __ldg(reinterpret_cast<const float4 *>(src + slice * CH));
+                e[0] = q.x; e[1] = q.y; e[CH - 2] = q.z; e[CH - 1] = q.w;
+            } else {
+#pragma unroll
+                for (int i = 0; i < CH; ++i) e[i] = __ldg(src + slice_element<CH, ROPE>(s.layout, slice, i));
+            }
+            if (CH == 4) *reinterpret_cast<float4 *>(dst) = make_float4(e[0], e[1], e[CH - 2], e[CH - 1]);
+            else {
+#pragma unroll
+                for (int i = 0; i < CH; ++i) dst[i] = e[i];
+            }
         }
     } else {
         const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256) + (size_t)slice * s.K * CH;

@@ -452,39 +452,48 @@ decode_rope_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__re
     decode_sliced_body<DT, 4, true, ROPE>(s, codes, std16, n, nullptr, cb, out, stride, st, table, ra);
 }
 
-// Any other shape: one thread per (head vector, pair of channels), codeword entries gathered from
-// global memory, float32 sums in stage order, rotation, one rounding.
+// Any other shape: a block decodes a few head vectors into shared memory (one thread per group row and
+// four-element piece: float4 gathers of the float32 codebooks, float32 sums in stage order), then one thread
+// per pair of channels rotates and stores.
 __global__ void __launch_bounds__(256)
 decode_rope_gather_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
                           const float *__restrict__ cb, void *__restrict__ out, int64_t stride, rvq_status *st,
-                          RopeArgs ra, int style)
+                          RopeArgs ra, int style, int vpb)
 {
-    const int half = s.dim / 2;
-    const int64_t total = n * half;
-    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < total; t += (int64_t)gridDim.x * 256) {
-        const int64_t v = t / half;
-        const int f = (int)(t - v * half);
-        const int c0 = style == 1 ? f : 2 * f, c1 = style == 1 ? f + half : 2 * f + 1;
-        const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes;
-        float val[2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int c = h ? c1 : c0;
-            const int g = s.layout == RVQ_GROUP_STRIDED ? c % s.G : c / s.gd;
-            const int i = s.layout == RVQ_GROUP_STRIDED ? c / s.G : c % s.gd;
-            float acc = 0.0f;
+    extern __shared__ __align__(16) float xs[];                   // [vpb][dim]
+    const int pieces = s.gd / 4, per_vec = s.G * pieces, half = s.dim / 2;
+    for (int64_t v0 = (int64_t)blockIdx.x * vpb; v0 < n; v0 += (int64_t)gridDim.x * vpb) {
+        for (int t = threadIdx.x; t < vpb * per_vec; t += 256) {
+            const int vl = t / per_vec, rem = t - vl * per_vec, g = rem / pieces, q = rem - g * pieces;
+            const int64_t v = v0 + vl;
+            if (v >= n) continue;
+            const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int r = 0; r < s.R; ++r) {
                 uint32_t j = read_code(vec, g * s.R + r, s.bits, s.code_bytes);
-                if (j >= (uint32_t)s.K) { j = 0; if (st && i == 0) atomicAdd(&st->bad_codes, 1u); }
-                acc += __ldg(cb + ((size_t)r * s.K + j) * s.gd + i);
+                if (j >= (uint32_t)s.K) { j = 0; if (st && q == 0) atomicAdd(&st->bad_codes, 1u); }
+                const float4 e = __ldg(reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * s.gd) + q);
+                acc.x += e.x; acc.y += e.y; acc.z += e.z; acc.w += e.w;
             }
-            val[h] = acc * __half2float(__ushort_as_half(std16[v]));
+            const float sd = __half2float(__ushort_as_half(std16[v]));
+            const float o[4] = {sd * acc.x, sd * acc.y, sd * acc.z, sd * acc.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) xs[vl * s.dim + channel_of(s.layout, s.G, s.gd, g, 4 * q + k)] = o[k];
         }
-        int pos = ra.position[v / ra.per_position];
-        pos = min(max(pos, 0), ra.positions - 1);
-        const float2 cs = __ldg(ra.table + (size_t)pos * half + f);
-        store_from_float(out, v * stride + c0, s.dtype, val[0] * cs.x - val[1] * cs.y);
-        store_from_float(out, v * stride + c1, s.dtype, val[1] * cs.x + val[0] * cs.y);
+        __syncthreads();
+        for (int t = threadIdx.x; t < vpb * half; t += 256) {
+            const int vl = t / half, f = t - vl * half;
+            const int64_t v = v0 + vl;
+            if (v >= n) continue;
+            const int c0 = style == 1 ? f : 2 * f, c1 = style == 1 ? f + half : 2 * f + 1;
+            int pos = ra.position[v / ra.per_position];
+            pos = min(max(pos, 0), ra.positions - 1);
+            const float2 cs = __ldg(ra.table + (size_t)pos * half + f);
+            const float a = xs[vl * s.dim + c0], b = xs[vl * s.dim + c1];
+            store_from_float(out, v * stride + c0, s.dtype, a * cs.x - b * cs.y);
+            store_from_float(out, v * stride + c1, s.dtype, b * cs.x + a * cs.y);
+        }
+        __syncthreads();
     }
 }
 
@@ -518,11 +527,14 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     if (n == 0) return RVQ_OK;
     RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions};
     if (!decode_exact_tables(s) || n > 0x7FFFFFFF) {
-        const int64_t total = n * (s.dim / 2);
-        int64_t blocks = (total + 255) / 256;
-        if (blocks > 148 * 32) blocks = 148 * 32;
-        decode_rope_gather_kernel<<<(unsigned)blocks, 256, 0, stream>>>(s, codes, std16, n, cb, out, stride, st, ra,
-                                                                        style == 0 ? 1 : 2);
+        const int per_vec = s.G * (s.gd / 4);
+        int vpb = 256 / per_vec;
+        if (vpb < 1) vpb = 1;
+        int64_t blocks = (n + vpb - 1) / vpb;
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        const size_t smem = (size_t)vpb * s.dim * sizeof(float);
+        decode_rope_gather_kernel<<<(unsigned)blocks, 256, smem, stream>>>(s, codes, std16, n, cb, out, stride, st, ra,
+                                                                           style == 0 ? 1 : 2, vpb);
         return check_launch();
     }
     int dev = 0, sms = 0;

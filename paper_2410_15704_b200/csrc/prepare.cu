@@ -36,37 +36,44 @@ size_t prepared_bytes(const Shape &s)
     return (b + 255) / 256 * 256;
 }
 
-// One thread per (channel octet, code): 8 stages x 8 channels of levels, stored as one 16-byte
+// One thread per (channel octet, code, stage): 8 channels of levels, stored as one 16-byte
 // entry of a wide slice or as the 8-byte entries of two narrow slices.
 __global__ void __launch_bounds__(256)
 decode_table_kernel(Shape s, const float *__restrict__ cb, const DecodeParams *__restrict__ dp,
                     const float *__restrict__ lo, uint4 *__restrict__ table)
 {
-    const int j = blockIdx.x * 256 + threadIdx.x, octet = blockIdx.y;
+    const int t = blockIdx.x * 256 + threadIdx.x, octet = blockIdx.y;
+    const int j = t >> 3, r = t & 7;
     if (j >= s.K) return;
     const bool wide = decode_slice_channels(s.K) == 8;
-    for (int r = 0; r < 8; ++r) {
-        uint32_t w[4];
-        for (int c = 0; c < 4; ++c) {
-            uint32_t pair = 0;
-            for (int h = 0; h < 2; ++h) {
-                uint32_t level = 0;
-                if (r < s.R && dp->step[r] > 0.0f) {
-                    const float v = cb[((size_t)r * s.K + j) * 32 + octet * 8 + 2 * c + h];
-                    const float q = rintf((v - lo[r]) / dp->step[r] * 32768.0f);
-                    level = (uint32_t)fminf(fmaxf(q, 0.0f), 32767.0f);
-                }
-                pair |= (0x8000u | level) << (16 * h);
+    const bool used = r < s.R && dp->step[r] > 0.0f;
+    float v[8];
+    if (used) {
+        const float4 *src = reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * 32 + octet * 8);
+        const float4 a = __ldg(src), b = __ldg(src + 1);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    }
+    uint32_t w[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint32_t pair = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t level = 0;
+            if (used) {
+                const float q = rintf((v[2 * c + h] - lo[r]) / dp->step[r] * 32768.0f);
+                level = (uint32_t)fminf(fmaxf(q, 0.0f), 32767.0f);
             }
-            w[c] = pair;
+            pair |= (0x8000u | level) << (16 * h);
         }
-        if (wide) {
-            table[((size_t)octet * s.K + j) * 8 + r] = make_uint4(w[0], w[1], w[2], w[3]);
-        } else {
-            uint2 *t2 = reinterpret_cast<uint2 *>(table);
-            t2[((size_t)(2 * octet) * s.K + j) * 8 + r] = make_uint2(w[0], w[1]);
-            t2[((size_t)(2 * octet + 1) * s.K + j) * 8 + r] = make_uint2(w[2], w[3]);
-        }
+        w[c] = pair;
+    }
+    if (wide) {
+        table[((size_t)octet * s.K + j) * 8 + r] = make_uint4(w[0], w[1], w[2], w[3]);
+    } else {
+        uint2 *t2 = reinterpret_cast<uint2 *>(table);
+        t2[((size_t)(2 * octet) * s.K + j) * 8 + r] = make_uint2(w[0], w[1]);
+        t2[((size_t)(2 * octet + 1) * s.K + j) * 8 + r] = make_uint2(w[2], w[3]);
     }
 }
 
@@ -248,7 +255,7 @@ int launch_prepare(const Shape &s, const float *cb, void *prepared, cudaStream_t
         if ((rc = check_launch()) != RVQ_OK) return rc;
     }
     if (dec) {
-        dim3 grid((s.K + 255) / 256, 4);
+        dim3 grid((s.K * 8 + 255) / 256, 4);
         decode_table_kernel<<<grid, 256, 0, stream>>>(s, cb, dp, lo, reinterpret_cast<uint4 *>(p + off + 256));
         if ((rc = check_launch()) != RVQ_OK) return rc;
     }

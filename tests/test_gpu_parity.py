@@ -215,6 +215,26 @@ def test_tensor_encode_equals_exact_encode():
         assert st["wait_timeouts"] == 0 and st["exhaustive_rows"] < 1e-3 * rows
 
 
+@pytest.mark.parametrize("name,tokens", [("ema_learning", 131072), ("value_cache", 32768)])
+def test_tensor_encode_equals_exact_encode_at_full_size(name, tokens):
+    """Tens of millions of (row, stage) choices at the sizes the timings are quoted on: the error
+    window of the tensor-core scores (prepare.cu) must never have hidden the exact winner."""
+    w = rvq_synth.WORKLOADS[name](tokens)
+    cfg = config_of(w)
+    xd = x_to_device(w.x, cfg.x_dtype)
+    b = rvq.alloc_buffers(cfg, w.n, w.codebooks)
+    exact = torch.empty_like(b.codes)
+    rvq.rvq_encode(cfg, xd, w.n, w.dim, b.codebooks, b.prepared, b.codes, b.std, b.workspace, b.workspace_bytes,
+                   b.status)
+    rvq.rvq_encode_exact(cfg, xd, w.n, w.dim, b.codebooks, b.prepared, exact, b.std, b.status)
+    torch.cuda.synchronize()
+    differing = int((b.codes != exact).sum().item())
+    assert differing == 0, f"{differing} code bytes differ between the tensor-core and the float32 encode"
+    st = rvq.read_status(b.status)
+    assert st["wait_timeouts"] == 0
+    print(f"{name}: {w.n * w.groups * w.depth} row-stages identical, re-scored {st['rescored_rows']}")
+
+
 def test_fused_encode_stats_equals_encode_then_stats():
     """rvq_encode_stats gives rvq_encode's codes and rvq_ema_stats' counts and sums."""
     for w in (rvq_synth.key_cache(tokens=700), rvq_synth.tiny(1000)):

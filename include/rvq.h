@@ -167,9 +167,9 @@ int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n,
  * in float32 and rounded once to x_dtype.  For dim 128 = 4 groups of 32 with
  * depth <= 8 the codebook entries are read from shared-memory tables: float32
  * copies (up to 1792 codes per stage) or, for 16-bit outputs and up to 3072
- * codes, 15-bit levels of each stage's value range kept in the prepared block.
+ * codes, 16-bit levels of each stage's value range kept in the prepared block.
  * With the levels the sum before the multiplication by std is within
- * err = sum_r (max C_r - min C_r) * 2^-16 of the float32 one; a head vector whose
+ * err <= 1.04 * sum_r (max C_r - min C_r) * 2^-17 of the float32 one; a head vector whose
  * std would make std * err exceed 0.9e-3 gets the float32 sum instead, so the
  * value before the final rounding is always within 1e-3 of the exact one.  Other
  * shapes gather the float32 codebooks from global memory.

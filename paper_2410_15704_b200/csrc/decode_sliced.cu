@@ -5,7 +5,7 @@
 // 256 output bytes gathers 1024 table entries: the gather, not HBM, is the
 // limit, and it has to come from shared memory without bank conflicts.
 //   - A CTA keeps one channel slice (CH = 8 of the 32 codeword channels, 4 when
-//     there are more than 1536 codes per stage) of all stages as 15-bit levels:
+//     there are more than 1536 codes per stage) of all stages as 16-bit levels:
 //     16 CH bytes per code = 8 stages x 2 CH bytes.  The 32 / CH slices of a row
 //     tile are handled by as many CTAs; the codes they share come from L2.
 //   - One thread produces the CH channels of one (group row, slice).  It reads
@@ -13,11 +13,12 @@
 //     visits the stages in an order rotated by its lane, so with CH = 8 the 8
 //     lanes of a quarter warp always touch 8 different 16-byte bank groups
 //     whatever the codes are (with CH = 4 two lanes of a half warp can meet).
-//   - A level q becomes the float 1 + q 2^-15 by one byte permute (the stored
-//     level carries the exponent's low bit), and one packed float32x2 FMA with
-//     the stage's step adds two channels to their float32 sums, which start at
-//     the affine offset of all stages; the sums are then multiplied by the
-//     stored deviation and rounded once.
+//   - A table entry is a 16-bit level q of its stage's value range, whose unit is
+//     an integer multiple (1..255) of a base common to all stages.  One 16-bit x
+//     8-bit dot-product instruction per channel and stage accumulates q * scale
+//     exactly in 32-bit integers; the sum is converted once, mapped back with the
+//     base and the sum of the stage minima, multiplied by the stored deviation
+//     and rounded once.
 //   - The level tables are off by at most dp->err (half a level per stage) times
 //     the deviation.  A row whose deviation makes that more than 0.9e-3 sums the
 //     float32 codewords instead (stage order, from global memory), so the result
@@ -48,28 +49,6 @@ template <> struct Out<RVQ_F16> {
     }
 };
 
-// Float 1 + q * 2^-15 from the low (H = 0) or high (H = 1) half of a table word.
-template <int H>
-__device__ __forceinline__ float level_to_float(uint32_t word)
-{
-    // bytes of the result, most significant first: 0x3F, half's high byte, half's low byte, 0x00
-    return __uint_as_float(__byte_perm(word, 0x3F000000u, H ? 0x7324 : 0x7104));
-}
-
-// Packed float32x2 multiply-add (one instruction for two channels).
-__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
-{
-    float2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;"
-        : "=l"(*reinterpret_cast<unsigned long long *>(&d))
-        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)),
-          "l"(*reinterpret_cast<unsigned long long *>(&c)));
-    return d;
-}
-
-// F32T: the tables hold the float32 codebook entries themselves (16 bytes per stage with
-// CH = 4: the same shared-memory geometry as the 15-bit tables with CH = 8) and the sums are
-// exact float32 sums; otherwise 15-bit levels as described above.
 // Codes r = 0 .. R-1 (R <= 8) of BITS bits each (BITS = 0: `bits`, known at run time only) from the 96-bit
 // window u0:u1:u2, packed two per word into cw[4] (which comes in zeroed).
 template <int BITS, bool FULL = false>      // FULL: R is 8
@@ -153,11 +132,11 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
         for (int t = tid; t < s.K * CH; t += kDecThreads) dst[t] = __ldg(src + t);
     }
     // this thread visits stage (rot + k) & 7 at step k: its steps' scales and line offsets
-    float step[8];
+    uint32_t scale[8];
     uint32_t unit[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { step[k] = F32T ? 0.0f : dp->step[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * kEntry; }
-    const float bias = F32T ? 0.0f : dp->bias;
+    for (int k = 0; k < 8; ++k) { scale[k] = F32T ? 0u : dp->scale[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * kEntry; }
+    const float bias = F32T ? 0.0f : dp->bias, base = F32T ? 0.0f : dp->base;
     const float exact_above = F32T ? INFINITY : (dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY);   // deviations the tables may serve
     __syncthreads();
 
@@ -269,14 +248,15 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
 #pragma unroll
             for (int i = 0; i < CH; ++i) o8[i] = acc[i] * sd;
         } else {
-            // two channels per packed float32x2 accumulator, started at the affine offset
-            float2 acc[CH / 2];
+            // integer sums of level * scale: one 16-bit x 8-bit dot-product instruction per channel and stage
+            // (the scale sits in byte 0 for the low half of a table word, in byte 1 for the high half)
+            uint32_t acc[CH];
 #pragma unroll
-            for (int i = 0; i < CH / 2; ++i) acc[i] = make_float2(bias, bias);
+            for (int i = 0; i < CH; ++i) acc[i] = 0u;
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const uint32_t j = (k & 1) ? (cw[k >> 1] >> 16) : (cw[k >> 1] & 0xFFFFu);
-                const float2 sk = make_float2(step[k], step[k]);
+                const uint32_t s_lo = scale[k], s_hi = scale[k] << 8;
                 uint32_t e[CH / 2];
                 if (CH == 8) {
                     const uint4 t = *reinterpret_cast<const uint4 *>(table + j * kLine + unit[k]);
@@ -286,11 +266,13 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                     e[0] = t.x; e[1] = t.y;
                 }
 #pragma unroll
-                for (int i = 0; i < CH / 2; ++i)
-                    acc[i] = fma2(make_float2(level_to_float<0>(e[i]), level_to_float<1>(e[i])), sk, acc[i]);
+                for (int i = 0; i < CH / 2; ++i) {
+                    acc[2 * i] = __dp2a_lo(e[i], s_lo, acc[2 * i]);
+                    acc[2 * i + 1] = __dp2a_lo(e[i], s_hi, acc[2 * i + 1]);
+                }
             }
 #pragma unroll
-            for (int i = 0; i < CH / 2; ++i) { o8[2 * i] = acc[i].x * sd; o8[2 * i + 1] = acc[i].y * sd; }
+            for (int i = 0; i < CH; ++i) o8[i] = fmaf((float)acc[i], base, bias) * sd;
         }
         if (!F32T && fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
             // too coarse for this deviation: the float32 codewords themselves, summed in stage order

@@ -61,10 +61,10 @@ decode_table_kernel(Shape s, const float *__restrict__ cb, const DecodeParams *_
         for (int h = 0; h < 2; ++h) {
             uint32_t level = 0;
             if (used) {
-                const float q = rintf((v[2 * c + h] - lo[r]) / dp->step[r] * 32768.0f);
-                level = (uint32_t)fminf(fmaxf(q, 0.0f), 32767.0f);
+                const float q = rintf((v[2 * c + h] - lo[r]) / dp->step[r]);
+                level = (uint32_t)fminf(fmaxf(q, 0.0f), 65535.0f);
             }
-            pair |= (0x8000u | level) << (16 * h);
+            pair |= level << (16 * h);
         }
         w[c] = pair;
     }
@@ -141,7 +141,7 @@ prepare_params_kernel(Shape s, const StagePartial *__restrict__ part, PreparedHe
         sp[r].b = INFINITY;
         sp[r].unsafe = (!isfinite(maxn) || ldexp(maxn, 2 * k) > 8200.0) ? 1.0f : 0.0f;
         mx[r].emax = 0u; mx[r].eerr = 0u; mx[r].nmax = 0u; mx[r].elomax = 0u;
-        if (r < 8) { s_lo[r] = lo; s_step[r] = hi > lo ? (hi - lo) * (32768.0f / 32767.0f) : 0.0f; }
+        if (r < 8) { s_lo[r] = lo; s_step[r] = hi > lo ? (hi - lo) / 65535.0f : 0.0f; }     // finest unit the range allows
     }
     __syncwarp();
     if (r == 0) {
@@ -150,12 +150,22 @@ prepare_params_kernel(Shape s, const StagePartial *__restrict__ part, PreparedHe
         hdr->decode_offset = decode_levels_prepared(s)
             ? (uint32_t)((kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256) : 0u;
         if (dp) {
+            // a common base and integer scales 1..255: the unit of a stage becomes scale * base >= its finest
+            float umax = 0.0f;
+            for (int q = 0; q < 8; ++q) umax = fmaxf(umax, s_step[q]);
+            const float base = umax / 255.0f;
             float b = 0.0f, e = 0.0f;
             for (int q = 0; q < 8; ++q) {
-                dp->step[q] = s_step[q]; dec_lo[q] = s_lo[q];
-                b += s_lo[q] - s_step[q]; e += s_step[q] * 1.52587890625e-5f;       // half a level per stage
+                uint32_t sc = 0;
+                if (s_step[q] > 0.0f) {
+                    sc = (uint32_t)fminf(255.0f, ceilf(s_step[q] / base));
+                    while (sc < 255u && (float)sc * base < s_step[q]) ++sc;       // (rounding of the division)
+                }
+                dp->scale[q] = sc;
+                dp->step[q] = (float)sc * base; dec_lo[q] = s_lo[q];
+                b += s_lo[q]; e += 0.5f * (float)sc * base * 1.0001f;             // half a level per stage
             }
-            dp->bias = b; dp->err = e;
+            dp->bias = b; dp->err = e; dp->base = base;
         }
     }
 }

@@ -22,17 +22,20 @@ struct PreparedHeader {
 };
 
 // Decoder section (group_dim 32, R <= 8, K <= kDecodeMaxK): per stage an affine
-// map value = lo + (f - 1) * step with f = 1 + q * 2^-15 in [1, 2) the float whose
-// mantissa bits 22..8 are the 15-bit level q, then channel slices of the
-// codebooks as levels: table[slice][code][stage 0..7][CH channels] uint16, each
-// with bit 15 set (it becomes the lowest exponent bit of f).  A slice is CH = 8
+// map value = lo_r + q * scale_r * base with q a 16-bit level, scale_r an integer in
+// 1..255 and base common to all stages, so that the sum over the stages is
+// sum lo_r + base * (sum q_r scale_r) with the second sum exact in 32-bit integers
+// (at most 8 * 65535 * 255); then channel slices of the codebooks as levels:
+// table[slice][code][stage 0..7][CH channels] uint16.  A slice is CH = 8
 // channels wide (four slices) while K <= kDecodeWideK and 4 channels (eight
 // slices) above, so that one slice of all codes fits the shared memory of a CTA.
 struct DecodeParams {
-    float step[8];    // (max - min) * 32768 / 32767 per stage, 0 for absent stages
-    float bias;       // sum over stages of (min - step)
-    float err;        // bound on |sum of table values - sum of float32 values| per channel
-    float pad[6];
+    float step[8];     // value of one level, scale_r * base, per stage; 0 for absent stages
+    float bias;        // sum over stages of the stage minimum lo_r
+    float err;         // bound on |sum of table values - sum of float32 values| per channel
+    float base;
+    float pad[5];
+    uint32_t scale[8]; // integer scale of a stage's levels (0 for absent stages)
 };
 constexpr int kDecodeWideK = 1536;                        // 128 bytes per code per slice in shared memory
 constexpr int kDecodeMaxK = 3072;                         // 64 bytes per code per slice
@@ -41,7 +44,7 @@ __host__ __device__ inline size_t decode_table_bytes(int K) { return (size_t)K *
 constexpr int kDecodeExactK = 1792;                       // float32 tables: 128 bytes per code per 4-channel slice
 // Which decoder serves a shape (group_dim 32, dim 128, depth <= 8; everything else gathers from global memory):
 //   - float32 table slices (exact sums, any output type) fit shared memory up to kDecodeExactK codes;
-//   - 15-bit level tables (16-bit outputs only: their own rounding, 2^-9 or 2^-12 relative, dwarfs the
+//   - 16-bit level tables (16-bit outputs only: their own rounding, 2^-9 or 2^-12 relative, dwarfs the
 //     tables') fit up to kDecodeMaxK codes and are the faster ones while the deviations are moderate;
 //   - up to kDecodeWideK codes and 16-bit outputs both fit, and the kernel chooses from the deviations.
 __host__ __device__ inline bool decode_exact_tables(const Shape &s)

@@ -195,13 +195,18 @@ int rvq_decode(const rvq_config *cfg /* host */, const void *codes, const uint16
  *                             values outside [0, positions) are clamped into it
  *   cos_sin               in  device float32 [positions][dim/2][2], 16-byte aligned, e.g. from
  *                             rvq_rope_table
- * dim 128 in 4 groups of 32, depth <= 8 and up to 1792 codes per stage use float32
- * shared-memory tables (exact float32 sums); other shapes gather from global memory.
+ *   prepared              in  block of rvq_prepare_codebooks for these codebooks, or NULL
+ * dim 128 in 4 groups of 32 with depth <= 8: up to 1792 codes per stage float32
+ * shared-memory tables (exact float32 sums); up to 3072 codes, 16-bit outputs and a
+ * prepared block, the level tables described under rvq_decode (a head vector whose
+ * std would make std * err exceed 0.6e-3 gets float32 sums instead, so the rotated
+ * value before the final rounding stays within 1e-3 of the exact one).  Other shapes,
+ * and these without a prepared block, gather from global memory.
  */
 enum { RVQ_ROPE_HALVES = 0, RVQ_ROPE_ADJACENT = 1 };
 int rvq_decode_rope(const rvq_config *cfg /* host */, const void *codes, const uint16_t *std_f16,
-                    int64_t n, const float *codebooks, const int32_t *position,
-                    int32_t vectors_per_position, const float *cos_sin, int32_t positions,
+                    int64_t n, const float *codebooks, const void *prepared,
+                    const int32_t *position, int32_t vectors_per_position, const float *cos_sin, int32_t positions,
                     int32_t pairing, void *x_out, int64_t out_row_stride, rvq_status *status,
                     void *stream /* cudaStream_t */);
 

@@ -77,8 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.rvq_rope_table.restype = ctypes.c_int
     lib.rvq_rope_table.argtypes = [ctypes.c_int32, ctypes.c_double, ctypes.c_int32, vp, vp]
     lib.rvq_decode_rope.restype = ctypes.c_int
-    lib.rvq_decode_rope.argtypes = [cfgp, vp, vp, i64, vp, vp, ctypes.c_int32, vp, ctypes.c_int32, ctypes.c_int32,
-                                    vp, i64, vp, vp]
+    lib.rvq_decode_rope.argtypes = [cfgp, vp, vp, i64, vp, vp, vp, ctypes.c_int32, vp, ctypes.c_int32,
+                                    ctypes.c_int32, vp, i64, vp, vp]
     lib.rvq_learn_step.restype = ctypes.c_int
     lib.rvq_learn_step.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
                                    vp, sz, vp, vp]
@@ -238,10 +238,11 @@ def rvq_rope_table(dim, base, positions, cos_sin, stream=None, check=True) -> in
     return rc
 
 
-def rvq_decode_rope(cfg, codes, std_f16, n, codebooks, position, vectors_per_position, cos_sin, positions,
-                    pairing, x_out, out_row_stride, status=None, stream=None, check=True) -> int:
-    """Decode and rotate: x_out = RoPE(decode(codes)) at the given positions."""
-    rc = lib.rvq_decode_rope(ctypes.byref(cfg), _ptr(codes), _ptr(std_f16), n, _ptr(codebooks), _ptr(position),
+def rvq_decode_rope(cfg, codes, std_f16, n, codebooks, prepared, position, vectors_per_position, cos_sin,
+                    positions, pairing, x_out, out_row_stride, status=None, stream=None, check=True) -> int:
+    """Decode and rotate: x_out = RoPE(decode(codes)) at the given positions (prepared may be None)."""
+    rc = lib.rvq_decode_rope(ctypes.byref(cfg), _ptr(codes), _ptr(std_f16), n, _ptr(codebooks), _ptr(prepared),
+                             _ptr(position),
                              vectors_per_position, _ptr(cos_sin), positions, pairing, _ptr(x_out), out_row_stride,
                              _ptr(status), _stream(stream))
     if check:

@@ -188,7 +188,8 @@ int rvq_rope_table(int32_t dim, double base, int32_t positions, float *cos_sin, 
 }
 
 int rvq_decode_rope(const rvq_config *cfg, const void *codes, const uint16_t *std_f16, int64_t n,
-                    const float *codebooks, const int32_t *position, int32_t vectors_per_position,
+                    const float *codebooks, const void *prepared, const int32_t *position,
+                    int32_t vectors_per_position,
                     const float *cos_sin, int32_t positions, int32_t pairing, void *x_out,
                     int64_t out_row_stride, rvq_status *status, void *stream)
 {
@@ -200,8 +201,8 @@ int rvq_decode_rope(const rvq_config *cfg, const void *codes, const uint16_t *st
     if (vectors_per_position < 1 || positions < 1 || (pairing != RVQ_ROPE_HALVES && pairing != RVQ_ROPE_ADJACENT))
         return RVQ_ERR_BADARG;
     if (s.dim & 1) return RVQ_ERR_UNSUPPORTED;
-    if (!aligned16(codebooks) || !aligned16(codes) || !aligned16(cos_sin)) return RVQ_ERR_ALIGN;
-    return launch_decode_rope(s, codes, std_f16, n, codebooks, position, vectors_per_position, cos_sin, positions,
+    if (!aligned16(codebooks) || !aligned16(codes) || !aligned16(cos_sin) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    return launch_decode_rope(s, codes, std_f16, n, codebooks, prepared, position, vectors_per_position, cos_sin, positions,
                               pairing, x_out, out_row_stride, status, (cudaStream_t)stream);
 }
 

@@ -42,8 +42,8 @@ int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std1
                          cudaStream_t stream);
 int launch_rope_table(int dim, double base, int positions, float *table, cudaStream_t stream);
 int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16, int64_t n, const float *cb,
-                       const int32_t *position, int per_position, const float *table, int positions, int style,
-                       void *out, int64_t stride, rvq_status *st, cudaStream_t stream);
+                       const void *prepared, const int32_t *position, int per_position, const float *table,
+                       int positions, int style, void *out, int64_t stride, rvq_status *st, cudaStream_t stream);
 int launch_ema_stats(const Shape &s, const void *x, int64_t n, int64_t stride, const void *codes,
                      const float *cb, float *batch_count, float *batch_sum, void *workspace,
                      rvq_status *st, cudaStream_t stream);

@@ -93,7 +93,7 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                    const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
                    int64_t stride, rvq_status *st, uint8_t *table, RopeArgs ra = RopeArgs())
 {
-    static_assert(ROPE == 0 || (F32T && CH == 4), "rotary decode uses float32 tables with 4-channel slices");
+    static_assert(ROPE == 0 || CH == 4, "rotary decode uses 4-channel slices");
     // table: [K][8 stages][kEntry bytes] in shared memory
     constexpr int NS = 32 / CH;                                  // slices
     if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;   // (a grid sized for another slice count)
@@ -126,6 +126,18 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                 for (int i = 0; i < CH; ++i) dst[i] = e[i];
             }
         }
+    } else if (ROPE != 0) {
+        // Level tables with the rotary slices: the prepared block keeps, per 4-element slice, entries of two
+        // words (elements 4s, 4s+1 | 4s+2, 4s+3); this CTA's entry takes the word of its places 0-1 and the
+        // word of its places 2-3, which for half-split pairs on strided groups come from two different slices.
+        const uint32_t *lev = reinterpret_cast<const uint32_t *>(dsec + 256);
+        const int ea = slice_element<CH, ROPE>(s.layout, slice, 0), eb = slice_element<CH, ROPE>(s.layout, slice, 2);
+        for (int t = tid; t < s.K * 8; t += kDecThreads) {
+            const int r = t & 7, j = t >> 3;
+            const uint32_t wa = __ldg(lev + ((((size_t)(ea >> 2) * s.K + j) * 8 + r) * 2 + ((ea & 3) >> 1)));
+            const uint32_t wb = __ldg(lev + ((((size_t)(eb >> 2) * s.K + j) * 8 + r) * 2 + ((eb & 3) >> 1)));
+            *reinterpret_cast<uint2 *>(table + (size_t)t * kEntry) = make_uint2(wa, wb);
+        }
     } else {
         const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256) + (size_t)slice * s.K * CH;
         uint4 *dst = reinterpret_cast<uint4 *>(table);
@@ -137,7 +149,8 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
 #pragma unroll
     for (int k = 0; k < 8; ++k) { scale[k] = F32T ? 0u : dp->scale[(rot + k) & 7]; unit[k] = (uint32_t)((rot + k) & 7) * kEntry; }
     const float bias = F32T ? 0.0f : dp->bias, base = F32T ? 0.0f : dp->base;
-    const float exact_above = F32T ? INFINITY : (dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY);   // deviations the tables may serve
+    // deviations the tables may serve (a rotation mixes two table values: their errors add up to sqrt(2) times one)
+    const float exact_above = F32T ? INFINITY : (dp->err > 0.0f ? (ROPE != 0 ? 0.6e-3f : 0.9e-3f) / dp->err : INFINITY);
     __syncthreads();
 
     const int64_t rows = n * 4;
@@ -284,11 +297,17 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                 if (r < s.R) {
                     uint32_t j = (r & 1) ? (cn[r >> 1] >> 16) : (cn[r >> 1] & 0xFFFFu);
                     if (j >= (uint32_t)s.K) j = 0;
-                    const float4 *e = reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * 32 + slice * CH);
+                    if (ROPE != 0) {
+                        const float *e = cb + ((size_t)r * s.K + j) * 32;
 #pragma unroll
-                    for (int q = 0; q < CH / 4; ++q) {
-                        const float4 t = __ldg(e + q);
-                        ex[4 * q] += t.x; ex[4 * q + 1] += t.y; ex[4 * q + 2] += t.z; ex[4 * q + 3] += t.w;
+                        for (int i = 0; i < CH; ++i) ex[i] += __ldg(e + slice_element<CH, ROPE>(s.layout, slice, i));
+                    } else {
+                        const float4 *e = reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * 32 + slice * CH);
+#pragma unroll
+                        for (int q = 0; q < CH / 4; ++q) {
+                            const float4 t = __ldg(e + q);
+                            ex[4 * q] += t.x; ex[4 * q + 1] += t.y; ex[4 * q + 2] += t.z; ex[4 * q + 3] += t.w;
+                        }
                     }
                 }
             }
@@ -424,14 +443,16 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
     decode_sliced_body<DT, CH, F32T>(s, codes, std16, n, dsec, cb, out, stride, st, table);
 }
 
-// Decode with the rotary embedding: float32 tables, 4-channel slices (dim 128, up to 1792 codes).
-template <int DT, int ROPE>
+// Decode with the rotary embedding, 4-channel slices (dim 128): float32 tables up to 1792 codes per stage,
+// 16-bit level tables (16-bit outputs) up to 3072.
+template <int DT, int ROPE, bool F32T>
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_rope_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
-                   const float *__restrict__ cb, void *__restrict__ out, int64_t stride, rvq_status *st, RopeArgs ra)
+                   const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
+                   int64_t stride, rvq_status *st, RopeArgs ra)
 {
     extern __shared__ __align__(128) uint8_t table[];
-    decode_sliced_body<DT, 4, true, ROPE>(s, codes, std16, n, nullptr, cb, out, stride, st, table, ra);
+    decode_sliced_body<DT, 4, F32T, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
 }
 
 // Any other shape: a block decodes a few head vectors into shared memory (one thread per group row and
@@ -503,12 +524,14 @@ int launch_rope_table(int dim, double base, int positions, float *table, cudaStr
 }
 
 int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16, int64_t n, const float *cb,
-                       const int32_t *position, int per_position, const float *table, int positions, int style,
-                       void *out, int64_t stride, rvq_status *st, cudaStream_t stream)
+                       const void *prepared, const int32_t *position, int per_position, const float *table,
+                       int positions, int style, void *out, int64_t stride, rvq_status *st, cudaStream_t stream)
 {
     if (n == 0) return RVQ_OK;
     RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions};
-    if (!decode_exact_tables(s) || n > 0x7FFFFFFF) {
+    const bool f32t = decode_exact_tables(s);
+    const bool levels = !f32t && prepared != nullptr && decode_levels_supported(s) && decode_slice_channels(s.K) == 4;
+    if ((!f32t && !levels) || n > 0x7FFFFFFF) {
         const int per_vec = s.G * (s.gd / 4);
         int vpb = 256 / per_vec;
         if (vpb < 1) vpb = 1;
@@ -523,7 +546,10 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return RVQ_ERR_DEVICE;
-    const size_t smem = (size_t)s.K * 128;
+    const size_t smem = (size_t)s.K * (f32t ? 128 : 64);
+    const uint8_t *dsec = nullptr;
+    if (levels)
+        dsec = reinterpret_cast<const uint8_t *>(prepared) + (kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256;
     const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
     int parts = sms / 8;
     if (parts > tiles) parts = (int)tiles;
@@ -531,20 +557,27 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     auto launch = [&](auto kernel) -> int {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return RVQ_ERR_LAUNCH;
-        kernel<<<parts * 8, kDecThreads, smem, stream>>>(s, codes, std16, n, cb, out, stride, st, ra);
+        kernel<<<parts * 8, kDecThreads, smem, stream>>>(s, codes, std16, n, dsec, cb, out, stride, st, ra);
         return check_launch();
     };
+    if (levels) {
+        if (style == 0)
+            return s.dtype == RVQ_BF16 ? launch(decode_rope_kernel<RVQ_BF16, 1, false>)
+                                       : launch(decode_rope_kernel<RVQ_F16, 1, false>);
+        return s.dtype == RVQ_BF16 ? launch(decode_rope_kernel<RVQ_BF16, 2, false>)
+                                   : launch(decode_rope_kernel<RVQ_F16, 2, false>);
+    }
     if (style == 0) {
         switch (s.dtype) {
-        case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 1>);
-        case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 1>);
-        default: return launch(decode_rope_kernel<RVQ_F16, 1>);
+        case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 1, true>);
+        case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 1, true>);
+        default: return launch(decode_rope_kernel<RVQ_F16, 1, true>);
         }
     }
     switch (s.dtype) {
-    case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 2>);
-    case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 2>);
-    default: return launch(decode_rope_kernel<RVQ_F16, 2>);
+    case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 2, true>);
+    case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 2, true>);
+    default: return launch(decode_rope_kernel<RVQ_F16, 2, true>);
     }
 }
 

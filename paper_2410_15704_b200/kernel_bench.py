@@ -124,7 +124,7 @@ def main():
                     table = torch.empty(max_pos, w.dim // 2, 2, device="cuda")
                     rvq.rvq_rope_table(w.dim, 500000.0, max_pos, table)
                     pos = (torch.arange(tokens, device="cuda", dtype=torch.int32) % max_pos).contiguous()
-                    med, best = timed(lambda: rvq.rvq_decode_rope(cfg, b.codes, b.std, n, b.codebooks, pos, w.heads,
+                    med, best = timed(lambda: rvq.rvq_decode_rope(cfg, b.codes, b.std, n, b.codebooks, b.prepared, pos, w.heads,
                                                                   table, max_pos, rvq.ROPE_HALVES, out, w.dim,
                                                                   b.status), args.reps, flush)
                     extra = w.dim // 2 * 8 // w.heads + 4 // w.heads      # a table row and a position per token

@@ -28,11 +28,12 @@ def test_rope_table_matches_double_precision():
     assert np.abs(t[:, :, 0] - np.cos(ang)).max() <= 1e-7 and np.abs(t[:, :, 1] - np.sin(ang)).max() <= 1e-7
 
 
-def run_case(dim, gd, R, K, bits, layout, dtype, pairing, tokens=333, heads=8, max_pos=100000):
+def run_case(dim, gd, R, K, bits, layout, dtype, pairing, tokens=333, heads=8, max_pos=100000, with_prepared=True,
+             std_scale=1.0):
     g = np.random.default_rng(dim + K + R + layout * 7 + pairing)
     n, G = tokens * heads, dim // gd
     codes = g.integers(0, K, size=(n, G, R)).astype(np.int32)
-    std_bits = (np.abs(1.0 + 0.25 * g.normal(size=n)) + 0.05).astype(np.float16).view(np.uint16)
+    std_bits = (std_scale * (np.abs(1.0 + 0.25 * g.normal(size=n)) + 0.05)).astype(np.float16).view(np.uint16)
     cb = np.stack([g.normal(scale=0.5 * 0.75 ** r, size=(K, gd)) for r in range(R)]).astype(np.float32)
     pos = g.integers(0, max_pos, size=tokens).astype(np.int32)
     pos[:3] = [0, max_pos - 1, 1]
@@ -40,9 +41,10 @@ def run_case(dim, gd, R, K, bits, layout, dtype, pairing, tokens=333, heads=8, m
     table = rope_table(dim, max_pos)
     out = torch.full((n, dim + 8), 7.0, dtype=rvq.TORCH_DTYPE[cfg.x_dtype], device="cuda")
     status = rvq.new_status()
+    b = rvq.alloc_buffers(cfg, n, cb)
     rvq.rvq_decode_rope(cfg, codes_to_device(cfg, codes), torch.from_numpy(std_bits.view(np.int16)).cuda(), n,
-                        torch.from_numpy(cb).cuda(), torch.from_numpy(pos).cuda(), heads, table, max_pos, pairing,
-                        out, dim + 8, status)
+                        b.codebooks, b.prepared if with_prepared else None, torch.from_numpy(pos).cuda(), heads, table,
+                        max_pos, pairing, out, dim + 8, status)
     torch.cuda.synchronize()
     got = out.float().cpu().numpy().astype(np.float64)
     assert np.all(got[:, dim:] == 7.0)                                   # row padding untouched
@@ -73,15 +75,26 @@ def test_decode_rope_table_path(layout, pairing, dtype):
 ])
 def test_decode_rope_other_shapes(dim, gd, R, K, bits, layout, dtype, pairing):
     run_case(dim, gd, R, K, bits, layout, dtype, pairing, tokens=97, heads=4, max_pos=5000)
+    run_case(dim, gd, R, K, bits, layout, dtype, pairing, tokens=97, heads=4, max_pos=5000, with_prepared=False)
+
+
+@pytest.mark.parametrize("layout", [rvq_synth.CONTIGUOUS, rvq_synth.STRIDED])
+@pytest.mark.parametrize("pairing", [rvq.ROPE_HALVES, rvq.ROPE_ADJACENT])
+def test_decode_rope_level_tables(layout, pairing):
+    """2048 and 3072 codes with 16-bit outputs: level tables; large deviations take float32 sums."""
+    run_case(128, 32, 8, 2048, 11, layout, "bf16", pairing, tokens=211)
+    run_case(128, 32, 8, 3072, 12, layout, "f16", pairing, tokens=57)
+    run_case(128, 32, 8, 2048, 16, layout, "bf16", pairing, tokens=57, std_scale=40.0)
 
 
 def test_decode_rope_clamps_positions_and_rejects_bad_arguments():
     import ctypes
     cfg = rvq.make_config(128, 32, 0, 8, 1024, 16, rvq.BF16, 0)
     c = ctypes.byref(cfg)
-    assert rvq.lib.rvq_decode_rope(c, 256, 256, 4, 256, 256, 0, 256, 10, 0, 256, 128, None, None) == -1   # 0 vectors per position
-    assert rvq.lib.rvq_decode_rope(c, 256, 256, 4, 256, 256, 8, 256, 10, 2, 256, 128, None, None) == -1   # unknown pairing
-    assert rvq.lib.rvq_decode_rope(c, 256, 256, 4, 256, None, 8, 256, 10, 0, 256, 128, None, None) == -1
+    assert rvq.lib.rvq_decode_rope(c, 256, 256, 4, 256, None, 256, 0, 256, 10, 0, 256, 128, None, None) == -1   # 0 vectors per position
+    assert rvq.lib.rvq_decode_rope(c, 256, 256, 4, 256, None, 256, 8, 256, 10, 2, 256, 128, None, None) == -1   # unknown pairing
+    assert rvq.lib.rvq_decode_rope(c, 256, 256, 4, 256, None, None, 8, 256, 10, 0, 256, 128, None, None) == -1
+    assert rvq.lib.rvq_decode_rope(c, 256, 256, 4, 256, 272, 256, 8, 256, 10, 0, 256, 128, None, None) == -2    # prepared % 256
     assert rvq.lib.rvq_rope_table(127, 10000.0, 4, 256, None) == -1
     # a position past the table reads its last row
     w = rvq_synth.decode_bandwidth(tokens=4)
@@ -91,7 +104,7 @@ def test_decode_rope_clamps_positions_and_rejects_bad_arguments():
         out = torch.empty(w.n, 128, dtype=torch.bfloat16, device="cuda")
         pos = torch.full((4,), p, dtype=torch.int32, device="cuda")
         rvq.rvq_decode_rope(cfg, codes_to_device(cfg, w.codes), torch.from_numpy(w.std_bits.view(np.int16)).cuda(),
-                            w.n, torch.from_numpy(w.codebooks).cuda(), pos, 8, table, 50, rvq.ROPE_HALVES, out, 128)
+                            w.n, torch.from_numpy(w.codebooks).cuda(), None, pos, 8, table, 50, rvq.ROPE_HALVES, out, 128)
         torch.cuda.synchronize()
         outs.append(out.cpu())
     assert torch.equal(outs[0], outs[1])

@@ -71,6 +71,7 @@ struct RopeArgs {
     int per_position;
     const float2 *table;          // (cos, sin) [positions][64]
     int positions;
+    int shift;                    // log2(per_position) when that is a power of two, else -1
 };
 
 // Codeword element held at place i of slice `slice`.
@@ -165,7 +166,7 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
         if (ROPE != 0) {
             // (the launcher sends larger problems elsewhere: a 64-bit division here is a subroutine call
             // that costs the whole loop its register allocation)
-            const uint32_t token = (uint32_t)v / (uint32_t)ra.per_position;
+            const uint32_t token = ra.shift >= 0 ? (uint32_t)v >> ra.shift : (uint32_t)v / (uint32_t)ra.per_position;
             int pos = live ? __ldg(ra.position + token) : 0;
             pos = min(max(pos, 0), ra.positions - 1);
             const float2 *cs = ra.table + (size_t)pos * 64;
@@ -528,7 +529,10 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
                        int positions, int style, void *out, int64_t stride, rvq_status *st, cudaStream_t stream)
 {
     if (n == 0) return RVQ_OK;
-    RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions};
+    int shift = -1;
+    for (int b = 0; b < 31; ++b)
+        if (per_position == (1 << b)) shift = b;
+    RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions, shift};
     const bool f32t = decode_exact_tables(s);
     const bool levels = !f32t && prepared != nullptr && decode_levels_supported(s) && decode_slice_channels(s.K) == 4;
     if ((!f32t && !levels) || n > 0x7FFFFFFF) {

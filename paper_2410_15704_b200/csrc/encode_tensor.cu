@@ -178,7 +178,7 @@ __device__ __forceinline__ float block_cells(const uint32_t (&u)[32], float (&t)
     for (int q = 0; q < 10; ++q)
         t[q] = min3(__uint_as_float(u[3 * q]), __uint_as_float(u[3 * q + 1]), __uint_as_float(u[3 * q + 2]));
     t[10] = fminf(__uint_as_float(u[30]), __uint_as_float(u[31]));
-    return fminf(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])), fminf(t[9], t[10]));
+    return min3(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])), t[9], t[10]);
 }
 
 // Keep a block's minimum if it is within the window of the running minimum.
@@ -530,7 +530,7 @@ encode_tensor_kernel(const Params p)
                     mbar_arrive(BAR(kBarAccFree + tile));        // the accumulator may be overwritten
                     const float c3 = block_cells(ub, t3);
 #pragma unroll
-                    for (int q = 0; q < 11; ++q) w.d[q] = fminf(min3(w.d[q], t0[q], t1[q]), fminf(t2[q], t3[q]));
+                    for (int q = 0; q < 11; ++q) w.d[q] = min3(min3(w.d[q], t0[q], t1[q]), t2[q], t3[q]);
                     list_block(w, c0, c * 4, list_v, list_i, kRowsPerPass);
                     list_block(w, c1, c * 4 + 1, list_v, list_i, kRowsPerPass);
                     list_block(w, c2, c * 4 + 2, list_v, list_i, kRowsPerPass);

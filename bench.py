@@ -386,7 +386,7 @@ def main():
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args)
     else:
-        args.steps = 1000 if args.steps is None else args.steps
+        args.steps = 3000 if args.steps is None else args.steps
         args.warmup = 5 if args.warmup is None else args.warmup
         run_ours(args)
 

@@ -301,6 +301,10 @@ def test_ragged_sizes(n):
     (128, 16, 8, 256, 1, "bf16", 8, 0),
     (128, 64, 3, 128, 0, "f32", 16, 0),
     (64, 8, 16, 64, 1, "f16", 6, 1),
+    (32, 32, 8, 512, 0, "bf16", 9, 0),          # one group per vector
+    (1024, 32, 2, 256, 1, "f32", 8, 0),         # 32 groups per vector: one vector per warp
+    (128, 32, 2, 4096, 0, "bf16", 12, 0),       # 32 operand slots per stage
+    (128, 32, 16, 128, 1, "bf16", 7, 0),        # the deepest stack
 ])
 def test_shape_grid(dim, gd, R, K, layout, dtype, bits, ddof):
     g = np.random.default_rng(dim + gd + R + K)

@@ -305,6 +305,8 @@ def test_ragged_sizes(n):
     (1024, 32, 2, 256, 1, "f32", 8, 0),         # 32 groups per vector: one vector per warp
     (128, 32, 2, 4096, 0, "bf16", 12, 0),       # 32 operand slots per stage
     (128, 32, 16, 128, 1, "bf16", 7, 0),        # the deepest stack
+    (128, 32, 1, 65536, 0, "bf16", 16, 0),      # the largest codebook the configuration admits
+    (128, 32, 2, 2, 1, "f32", 1, 0),            # and the smallest
 ])
 def test_shape_grid(dim, gd, R, K, layout, dtype, bits, ddof):
     g = np.random.default_rng(dim + gd + R + K)

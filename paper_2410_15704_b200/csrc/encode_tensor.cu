@@ -601,21 +601,6 @@ encode_tensor_kernel(const Params p)
                 // every listed block of one such row at a time (or all columns when the list
                 // overflowed), then reduces to the smallest distance, lowest index on ties.
                 uint32_t todo = __ballot_sync(0xFFFFFFFFu, flagged);
-                // first touch every codeword the loop below will read, so that their loads overlap
-                for (uint32_t pre = todo; pre; pre &= pre - 1) {
-                    const int src = __ffs(pre) - 1;
-                    const float lim_s = __shfl_sync(0xFFFFFFFFu, lim, src);
-                    const int cnt_s = __shfl_sync(0xFFFFFFFFu, cnt, src);
-                    const bool all_s = __shfl_sync(0xFFFFFFFFu, (int)scan_all, src) != 0;
-                    const int row_s = rloc - lane + src;
-                    if (all_s) continue;
-                    for (int e = 0; e < cnt_s; ++e) {
-                        const float fv = reinterpret_cast<const float *>(smem + kOffListV)[e * kRowsPerPass + row_s];
-                        if (!(fv <= lim_s)) continue;
-                        const int j = (int)reinterpret_cast<const uint16_t *>(smem + kOffListI)[e * kRowsPerPass + row_s] * 32 + lane;
-                        if (j < s.K) asm volatile("prefetch.global.L1 [%0];" ::"l"(cbr + (size_t)j * 32));
-                    }
-                }
                 while (todo) {
                     const int src = __ffs(todo) - 1;
                     todo &= todo - 1;

@@ -166,7 +166,7 @@ int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n,
  * channel c = channel(g, i): x_out[c] = std * sum_r C_r[code[g][r]][i], summed
  * in float32 and rounded once to x_dtype.  For dim 128 = 4 groups of 32 with
  * depth <= 8 the codebook entries are read from shared-memory tables: float32
- * copies (up to 1792 codes per stage) or, for 16-bit outputs and up to 3072
+ * copies (up to 3584 codes per stage) or, for 16-bit outputs and up to 3072
  * codes, 16-bit levels of each stage's value range kept in the prepared block.
  * With the levels the sum before the multiplication by std is within
  * err <= 1.04 * sum_r (max C_r - min C_r) * 2^-17 of the float32 one; a head vector whose
@@ -196,12 +196,12 @@ int rvq_decode(const rvq_config *cfg /* host */, const void *codes, const uint16
  *   cos_sin               in  device float32 [positions][dim/2][2], 16-byte aligned, e.g. from
  *                             rvq_rope_table
  *   prepared              in  block of rvq_prepare_codebooks for these codebooks, or NULL
- * dim 128 in 4 groups of 32 with depth <= 8: up to 1792 codes per stage float32
- * shared-memory tables (exact float32 sums); up to 3072 codes, 16-bit outputs and a
- * prepared block, the level tables described under rvq_decode (a head vector whose
- * std would make std * err exceed 0.6e-3 gets float32 sums instead, so the rotated
- * value before the final rounding stays within 1e-3 of the exact one).  Other shapes,
- * and these without a prepared block, gather from global memory.
+ * dim 128 in 4 groups of 32 with depth <= 8: up to 3584 codes per stage float32
+ * shared-memory tables (exact float32 sums); with 16-bit outputs, a prepared block and
+ * 1537..3072 codes also the level tables described under rvq_decode, chosen when the
+ * deviations are moderate (a head vector whose std would make std * err exceed 0.6e-3
+ * gets float32 sums, so the rotated value before the final rounding stays within 1e-3
+ * of the exact one).  Other shapes gather from global memory.
  */
 enum { RVQ_ROPE_HALVES = 0, RVQ_ROPE_ADJACENT = 1 };
 int rvq_decode_rope(const rvq_config *cfg /* host */, const void *codes, const uint16_t *std_f16,

@@ -78,7 +78,8 @@ struct RopeArgs {
 template <int CH, int ROPE>
 __device__ __forceinline__ int slice_element(int layout, int slice, int i)
 {
-    if (ROPE == 1 && layout == RVQ_GROUP_STRIDED) return 2 * slice + (i & 1) + 16 * (i >> 1);
+    if (ROPE == 1 && layout == RVQ_GROUP_STRIDED)       // the first CH / 2 places and their partners 16 elements on
+        return (CH / 2) * slice + (i % (CH / 2)) + 16 * (i / (CH / 2));
     return slice * CH + i;
 }
 
@@ -94,7 +95,8 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                    const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
                    int64_t stride, rvq_status *st, uint8_t *table, RopeArgs ra = RopeArgs())
 {
-    static_assert(ROPE == 0 || CH == 4, "rotary decode uses 4-channel slices");
+    static_assert(ROPE == 0 || CH == 4 || CH == 2, "rotary decode uses 4- or 2-channel slices");
+    static_assert(F32T || CH >= 4, "2-channel slices are for float32 tables");
     // table: [K][8 stages][kEntry bytes] in shared memory
     constexpr int NS = 32 / CH;                                  // slices
     if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;   // (a grid sized for another slice count)
@@ -113,15 +115,21 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
             if (r >= s.R) {
 #pragma unroll
                 for (int i = 0; i < CH; ++i) e[i] = 0.0f;
-            } else if (CH == 4 && slice_element<CH, ROPE>(s.layout, slice, 1) == slice * CH + 1 &&
+            } else if (CH == 4 && slice_element<CH, ROPE>(s.layout, slice, 0) == slice * CH &&
+                       slice_element<CH, ROPE>(s.layout, slice, 1) == slice * CH + 1 &&
                        slice_element<CH, ROPE>(s.layout, slice, 2) == slice * CH + 2) {
                 const float4 q = __ldg(reinterpret_cast<const float4 *>(src + slice * CH));
                 e[0] = q.x; e[1] = q.y; e[CH - 2] = q.z; e[CH - 1] = q.w;
+            } else if (CH == 2 && slice_element<CH, ROPE>(s.layout, slice, 0) == slice * CH &&
+                       slice_element<CH, ROPE>(s.layout, slice, 1) == slice * CH + 1) {
+                const float2 q = __ldg(reinterpret_cast<const float2 *>(src + slice * CH));
+                e[0] = q.x; e[1] = q.y;
             } else {
 #pragma unroll
                 for (int i = 0; i < CH; ++i) e[i] = __ldg(src + slice_element<CH, ROPE>(s.layout, slice, i));
             }
             if (CH == 4) *reinterpret_cast<float4 *>(dst) = make_float4(e[0], e[1], e[CH - 2], e[CH - 1]);
+            else if (CH == 2) *reinterpret_cast<float2 *>(dst) = make_float2(e[0], e[1]);
             else {
 #pragma unroll
                 for (int i = 0; i < CH; ++i) dst[i] = e[i];
@@ -170,7 +178,18 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
             int pos = live ? __ldg(ra.position + token) : 0;
             pos = min(max(pos, 0), ra.positions - 1);
             const float2 *cs = ra.table + (size_t)pos * 64;
-            if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) {          // pairs 4 (2 slice + i) + g
+            if (CH == 2) {
+                // one pair in the thread (half-split pairs on strided groups: pair 4 slice + g; adjacent pairs on
+                // contiguous groups: pair 16 g + slice), or two places whose partners sit in another lane
+                if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) rc[0] = __ldg(cs + slice * 4 + g);
+                else if (ROPE == 2 && s.layout != RVQ_GROUP_STRIDED) rc[0] = __ldg(cs + g * 16 + slice);
+                else if (ROPE == 1) {                                  // pairs 32 (g & 1) + 2 slice + i
+                    const float4 cc = __ldg(reinterpret_cast<const float4 *>(cs + (g & 1) * 32 + slice * 2));
+                    rc[0] = make_float2(cc.x, cc.y); rc[1] = make_float2(cc.z, cc.w);
+                } else {                                               // pairs 2 (2 slice + i) + g / 2
+                    rc[0] = __ldg(cs + slice * 4 + (g >> 1)); rc[1] = __ldg(cs + slice * 4 + 2 + (g >> 1));
+                }
+            } else if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) {   // pairs 4 (2 slice + i) + g
                 rc[0] = __ldg(cs + slice * 8 + g); rc[1] = __ldg(cs + slice * 8 + 4 + g);
             } else if (ROPE == 2 && s.layout != RVQ_GROUP_STRIDED) {   // pairs 16 g + 2 slice + i
                 const float4 cc = __ldg(reinterpret_cast<const float4 *>(cs + g * 16 + slice * 2));
@@ -244,7 +263,7 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
         }
         const float sd = live ? __half2float(__ushort_as_half(std16[v])) : 0.0f;
         float o8[CH];
-        if (F32T) {
+        if constexpr (F32T) {
             float acc[CH];
 #pragma unroll
             for (int i = 0; i < CH; ++i) acc[i] = 0.0f;
@@ -288,7 +307,7 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
 #pragma unroll
             for (int i = 0; i < CH; ++i) o8[i] = fmaf((float)acc[i], base, bias) * sd;
         }
-        if (!F32T && fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
+        if constexpr (!F32T) if (fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
             // too coarse for this deviation: the float32 codewords themselves, summed in stage order
             float ex[CH];
 #pragma unroll
@@ -318,18 +337,19 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
 
         if (ROPE != 0) {
             const bool strided = s.layout == RVQ_GROUP_STRIDED;
+            constexpr int H = CH / 2;
             if (ROPE == 1 && strided) {
-                // places 0, 1 are channels 4 e + g of the first half, places 2, 3 their partners 64 further on
+                // places 0 .. H-1 are channels 4 e + g of the first half, places H .. CH-1 their partners 64 further on
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const float a = o8[i], b = o8[i + 2];
+                for (int i = 0; i < H; ++i) {
+                    const float a = o8[i], b = o8[i + H];
                     o8[i] = a * rc[i].x - b * rc[i].y;
-                    o8[i + 2] = b * rc[i].x + a * rc[i].y;
+                    o8[i + H] = b * rc[i].x + a * rc[i].y;
                 }
             } else if (ROPE == 2 && !strided) {
-                // channels 32 g + 4 slice + i: pairs (0, 1) and (2, 3) are in this thread
+                // channels 32 g + CH slice + i: the pairs (0, 1) (and (2, 3)) are in this thread
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
+                for (int i = 0; i < H; ++i) {
                     const float a = o8[2 * i], b = o8[2 * i + 1];
                     o8[2 * i] = a * rc[i].x - b * rc[i].y;
                     o8[2 * i + 1] = b * rc[i].x + a * rc[i].y;
@@ -341,74 +361,104 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                 const int other = ROPE == 1 ? 2 : 1;
                 const bool first = (g & other) == 0;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < CH; ++i) {
                     const float b = __shfl_xor_sync(0xFFFFFFFFu, o8[i], other);
                     o8[i] = first ? o8[i] * rc[i].x - b * rc[i].y : o8[i] * rc[i].x + b * rc[i].y;
                 }
             }
         }
-        if (DT == RVQ_F32) {
-            if (s.layout == RVQ_GROUP_CONTIGUOUS) {
-                if (live) {
-                    float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + v * stride + g * 32 + slice * CH);
-#pragma unroll
-                    for (int i = 0; i < CH / 4; ++i)
-                        o[i] = make_float4(o8[4 * i], o8[4 * i + 1], o8[4 * i + 2], o8[4 * i + 3]);
+        if constexpr (CH == 2) {
+            // two places per thread
+            if (DT == RVQ_F32) {
+                float *o = reinterpret_cast<float *>(out) + v * stride;
+                if (s.layout == RVQ_GROUP_CONTIGUOUS) {
+                    if (live) *reinterpret_cast<float2 *>(o + g * 32 + slice * 2) = make_float2(o8[0], o8[1]);
+                } else if (live) {
+                    o[4 * slice_element<CH, ROPE>(s.layout, slice, 0) + g] = o8[0];
+                    o[4 * slice_element<CH, ROPE>(s.layout, slice, 1) + g] = o8[1];
                 }
-            } else if (live) {
-                float *o = reinterpret_cast<float *>(out) + v * stride + g;
-#pragma unroll
-                for (int i = 0; i < CH; ++i) o[4 * slice_element<CH, ROPE>(s.layout, slice, i)] = o8[i];   // channel 4 element + g
+            } else {
+                const uint32_t w0 = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(o8[0], o8[1]);
+                uint16_t *o16 = reinterpret_cast<uint16_t *>(out) + v * stride;
+                if (s.layout == RVQ_GROUP_CONTIGUOUS) {
+                    if (live) *reinterpret_cast<uint32_t *>(o16 + g * 32 + slice * 2) = w0;
+                } else {
+                    // Lane g holds places 0 and 1 of group g; the four lanes cover, per place, the four
+                    // consecutive channels 4 element .. 4 element + 3.  Lane L stores two of them: place L / 2,
+                    // groups 2 (L % 2) and 2 (L % 2) + 1, fetched from those two lanes.
+                    const int base_lane = (tid & 31) & ~3, ga = 2 * (g & 1);
+                    const uint32_t wa = __shfl_sync(0xFFFFFFFFu, w0, base_lane + ga);
+                    const uint32_t wb = __shfl_sync(0xFFFFFFFFu, w0, base_lane + ga + 1);
+                    const uint32_t both = __byte_perm(wa, wb, (g & 2) ? 0x7632 : 0x5410);
+                    if (live)
+                        *reinterpret_cast<uint32_t *>(o16 + 4 * slice_element<CH, ROPE>(s.layout, slice, g >> 1) + ga) = both;
+                }
             }
         } else {
-            uint32_t w[CH / 2];
-#pragma unroll
-            for (int c = 0; c < CH / 2; ++c) w[c] = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(o8[2 * c], o8[2 * c + 1]);
-            uint16_t *o16 = reinterpret_cast<uint16_t *>(out) + v * stride;
-            if (s.layout == RVQ_GROUP_CONTIGUOUS) {
-                if (live) {
-                    if (CH == 8)
-                        *reinterpret_cast<uint4 *>(o16 + g * 32 + slice * 8) = make_uint4(w[0], w[1], w[CH / 2 - 2], w[CH / 2 - 1]);
-                    else
-                        *reinterpret_cast<uint2 *>(o16 + g * 32 + slice * 4) = make_uint2(w[0], w[1]);
+            if (DT == RVQ_F32) {
+                if (s.layout == RVQ_GROUP_CONTIGUOUS) {
+                    if (live) {
+                        float4 *o = reinterpret_cast<float4 *>(reinterpret_cast<float *>(out) + v * stride + g * 32 + slice * CH);
+    #pragma unroll
+                        for (int i = 0; i < CH / 4; ++i)
+                            o[i] = make_float4(o8[4 * i], o8[4 * i + 1], o8[4 * i + 2], o8[4 * i + 3]);
+                    }
+                } else if (live) {
+                    float *o = reinterpret_cast<float *>(out) + v * stride + g;
+    #pragma unroll
+                    for (int i = 0; i < CH; ++i) o[4 * slice_element<CH, ROPE>(s.layout, slice, i)] = o8[i];   // channel 4 element + g
                 }
-            } else if (CH == 8) {
-                // Lane g holds element pairs (2c, 2c+1) of group g, i.e. channels 32 slice + 8c + g and + 4.
-                // Lane c' of the 4-lane set wants pairs c' of all four groups: a 4x4 transpose of words.
-                // two butterfly steps: exchange odd/even words with lane g^1, then word pairs with lane g^2
-                uint32_t &w0 = w[0], &w1 = w[1], &w2 = w[CH / 2 - 2], &w3 = w[CH / 2 - 1];
-                {
-                    const bool b1 = g & 1, b2 = g & 2;
-                    const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w0 : w1, 1);
-                    const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w2 : w3, 1);
-                    if (b1) { w0 = r0; w2 = r1; } else { w1 = r0; w3 = r1; }
-                    const uint32_t r2 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w0 : w2, 2);
-                    const uint32_t r3 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w1 : w3, 2);
-                    if (b2) { w0 = r2; w1 = r3; } else { w2 = r2; w3 = r3; }
-                }
-                // now w[q] = pair g of group q: (element 2g of group q, element 2g+1 of group q)
-                const uint32_t o0 = __byte_perm(w0, w1, 0x5410), o1 = __byte_perm(w2, w3, 0x5410);
-                const uint32_t o2 = __byte_perm(w0, w1, 0x7632), o3 = __byte_perm(w2, w3, 0x7632);
-                // channels 32 slice + 8 g + 0..7: element 2g of groups 0..3, then element 2g+1 of groups 0..3
-                if (live) *reinterpret_cast<uint4 *>(o16 + slice * 32 + g * 8) = make_uint4(o0, o1, o2, o3);
             } else {
-                // Lane g holds elements 4 slice + 0..3 of group g as w[0] = (e0, e1), w[1] = (e2, e3); the
-                // 16 channels 16 slice .. 16 slice + 15 are element-major, so lane L stores element L of
-                // the four groups.  Exchange words with lane g^2, then halves with lane g^1.
-                const bool b1 = g & 1, b2 = g & 2;
-                const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[0] : w[1], 2);
-                // lanes 0, 1 now hold (e0, e1) of groups g and g + 2; lanes 2, 3 hold (e2, e3) of g - 2 and g
-                const uint32_t lo_g = b2 ? r0 : w[0], hi_g = b2 ? w[1] : r0;   // lower and upper group of the pair
-                // keep the half this lane stores (e_L), send the other one
-                const uint32_t keep = __byte_perm(lo_g, hi_g, b1 ? 0x7632 : 0x5410);
-                const uint32_t send = __byte_perm(lo_g, hi_g, b1 ? 0x5410 : 0x7632);
-                const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
-                // keep = element L of groups (g & 1) and (g & 1) + 2, got = element L of the other two
-                const uint32_t even = b1 ? got : keep, odd = b1 ? keep : got;   // groups (0, 2) and (1, 3)
-                if (live)
-                    *reinterpret_cast<uint2 *>(o16 + 4 * slice_element<CH, ROPE>(s.layout, slice, g)) =
-                        make_uint2(__byte_perm(even, odd, 0x5410), __byte_perm(even, odd, 0x7632));
+                uint32_t w[CH / 2];
+    #pragma unroll
+                for (int c = 0; c < CH / 2; ++c) w[c] = Out<DT == RVQ_F32 ? RVQ_BF16 : DT>::pack(o8[2 * c], o8[2 * c + 1]);
+                uint16_t *o16 = reinterpret_cast<uint16_t *>(out) + v * stride;
+                if (s.layout == RVQ_GROUP_CONTIGUOUS) {
+                    if (live) {
+                        if (CH == 8)
+                            *reinterpret_cast<uint4 *>(o16 + g * 32 + slice * 8) = make_uint4(w[0], w[1], w[CH / 2 - 2], w[CH / 2 - 1]);
+                        else
+                            *reinterpret_cast<uint2 *>(o16 + g * 32 + slice * 4) = make_uint2(w[0], w[1]);
+                    }
+                } else if (CH == 8) {
+                    // Lane g holds element pairs (2c, 2c+1) of group g, i.e. channels 32 slice + 8c + g and + 4.
+                    // Lane c' of the 4-lane set wants pairs c' of all four groups: a 4x4 transpose of words.
+                    // two butterfly steps: exchange odd/even words with lane g^1, then word pairs with lane g^2
+                    uint32_t &w0 = w[0], &w1 = w[1], &w2 = w[CH / 2 - 2], &w3 = w[CH / 2 - 1];
+                    {
+                        const bool b1 = g & 1, b2 = g & 2;
+                        const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w0 : w1, 1);
+                        const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w2 : w3, 1);
+                        if (b1) { w0 = r0; w2 = r1; } else { w1 = r0; w3 = r1; }
+                        const uint32_t r2 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w0 : w2, 2);
+                        const uint32_t r3 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w1 : w3, 2);
+                        if (b2) { w0 = r2; w1 = r3; } else { w2 = r2; w3 = r3; }
+                    }
+                    // now w[q] = pair g of group q: (element 2g of group q, element 2g+1 of group q)
+                    const uint32_t o0 = __byte_perm(w0, w1, 0x5410), o1 = __byte_perm(w2, w3, 0x5410);
+                    const uint32_t o2 = __byte_perm(w0, w1, 0x7632), o3 = __byte_perm(w2, w3, 0x7632);
+                    // channels 32 slice + 8 g + 0..7: element 2g of groups 0..3, then element 2g+1 of groups 0..3
+                    if (live) *reinterpret_cast<uint4 *>(o16 + slice * 32 + g * 8) = make_uint4(o0, o1, o2, o3);
+                } else {
+                    // Lane g holds elements 4 slice + 0..3 of group g as w[0] = (e0, e1), w[1] = (e2, e3); the
+                    // 16 channels 16 slice .. 16 slice + 15 are element-major, so lane L stores element L of
+                    // the four groups.  Exchange words with lane g^2, then halves with lane g^1.
+                    const bool b1 = g & 1, b2 = g & 2;
+                    const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[0] : w[1], 2);
+                    // lanes 0, 1 now hold (e0, e1) of groups g and g + 2; lanes 2, 3 hold (e2, e3) of g - 2 and g
+                    const uint32_t lo_g = b2 ? r0 : w[0], hi_g = b2 ? w[1] : r0;   // lower and upper group of the pair
+                    // keep the half this lane stores (e_L), send the other one
+                    const uint32_t keep = __byte_perm(lo_g, hi_g, b1 ? 0x7632 : 0x5410);
+                    const uint32_t send = __byte_perm(lo_g, hi_g, b1 ? 0x5410 : 0x7632);
+                    const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+                    // keep = element L of groups (g & 1) and (g & 1) + 2, got = element L of the other two
+                    const uint32_t even = b1 ? got : keep, odd = b1 ? keep : got;   // groups (0, 2) and (1, 3)
+                    if (live)
+                        *reinterpret_cast<uint2 *>(o16 + 4 * slice_element<CH, ROPE>(s.layout, slice, g)) =
+                            make_uint2(__byte_perm(even, odd, 0x5410), __byte_perm(even, odd, 0x7632));
+                }
             }
+    
         }
     }
     if (bad && st && slice == 0) atomicAdd(&st->bad_codes, bad);   // every slice sees the same codes
@@ -417,10 +467,10 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
 // True when more than an eighth of a sample of up to 256 deviations is beyond the level tables' reach.
 // Uniform over the CTA (and over all CTAs of a launch: they read the same sample).
 __device__ __forceinline__ bool sample_wants_float32(const uint16_t *__restrict__ std16, int64_t n,
-                                                  const uint8_t *__restrict__ dsec)
+                                                  const uint8_t *__restrict__ dsec, float reach)
 {
     const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
-    const float exact_above = dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY;
+    const float exact_above = dp->err > 0.0f ? reach / dp->err : INFINITY;
     const int64_t samples = n < 256 ? n : 256, every = n < 256 ? 1 : n >> 8;
     const bool beyond = threadIdx.x < samples &&
                         fabsf(__half2float(__ushort_as_half(std16[threadIdx.x * every]))) > exact_above;
@@ -440,20 +490,21 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
                      int64_t stride, rvq_status *st)
 {
     extern __shared__ __align__(128) uint8_t table[];
-    if (PICK != 0 && sample_wants_float32(std16, n, dsec) != (PICK == 2)) return;
+    if (PICK != 0 && sample_wants_float32(std16, n, dsec, 0.9e-3f) != (PICK == 2)) return;
     decode_sliced_body<DT, CH, F32T>(s, codes, std16, n, dsec, cb, out, stride, st, table);
 }
 
 // Decode with the rotary embedding, 4-channel slices (dim 128): float32 tables up to 1792 codes per stage,
 // 16-bit level tables (16-bit outputs) up to 3072.
-template <int DT, int ROPE, bool F32T>
+template <int DT, int ROPE, int CH, bool F32T, int PICK>
 __global__ void __launch_bounds__(kDecThreads, 1)
 decode_rope_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
                    const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
                    int64_t stride, rvq_status *st, RopeArgs ra)
 {
     extern __shared__ __align__(128) uint8_t table[];
-    decode_sliced_body<DT, 4, F32T, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
+    if (PICK != 0 && sample_wants_float32(std16, n, dsec, 0.6e-3f) != (PICK == 2)) return;
+    decode_sliced_body<DT, CH, F32T, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
 }
 
 // Any other shape: a block decodes a few head vectors into shared memory (one thread per group row and
@@ -534,8 +585,8 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
         if (per_position == (1 << b)) shift = b;
     RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions, shift};
     const bool f32t = decode_exact_tables(s);
-    const bool levels = !f32t && prepared != nullptr && decode_levels_supported(s) && decode_slice_channels(s.K) == 4;
-    if ((!f32t && !levels) || n > 0x7FFFFFFF) {
+    const bool levels = prepared != nullptr && decode_levels_supported(s) && decode_slice_channels(s.K) == 4;
+    if (!f32t || n > 0x7FFFFFFF) {
         const int per_vec = s.G * (s.gd / 4);
         int vpb = 256 / per_vec;
         if (vpb < 1) vpb = 1;
@@ -550,39 +601,48 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return RVQ_ERR_DEVICE;
-    const size_t smem = (size_t)s.K * (f32t ? 128 : 64);
     const uint8_t *dsec = nullptr;
     if (levels)
         dsec = reinterpret_cast<const uint8_t *>(prepared) + (kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256;
     const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
-    int parts = sms / 8;
-    if (parts > tiles) parts = (int)tiles;
-    if (parts < 1) parts = 1;
-    auto launch = [&](auto kernel) -> int {
+    auto launch = [&](auto kernel, int ch, bool f32_tables) -> int {
+        const int ns = 32 / ch;
+        const size_t smem = (size_t)s.K * (f32_tables ? 32 : 16) * ch;
+        int parts = sms / ns;
+        if (parts > tiles) parts = (int)tiles;
+        if (parts < 1) parts = 1;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return RVQ_ERR_LAUNCH;
-        kernel<<<parts * 8, kDecThreads, smem, stream>>>(s, codes, std16, n, dsec, cb, out, stride, st, ra);
+        kernel<<<parts * ns, kDecThreads, smem, stream>>>(s, codes, std16, n, dsec, cb, out, stride, st, ra);
         return check_launch();
     };
+    // style 0/1 -> ROPE 1/2; float32 tables with 4-channel slices up to 1792 codes, 2-channel ones beyond; where
+    // level tables exist as well, both kernels are launched and the deviations decide on the device (PICK)
+    const bool wide = decode_exact_channels(s.K) == 4;
+#define RVQ_ROPE_F32(DT, PICK)                                                                                      \
+    (style == 0 ? (wide ? launch(decode_rope_kernel<DT, 1, 4, true, PICK>, 4, true)                                \
+                        : launch(decode_rope_kernel<DT, 1, 2, true, PICK>, 2, true))                               \
+                : (wide ? launch(decode_rope_kernel<DT, 2, 4, true, PICK>, 4, true)                                \
+                        : launch(decode_rope_kernel<DT, 2, 2, true, PICK>, 2, true)))
+#define RVQ_ROPE_LEVELS(DT)                                                                                         \
+    (style == 0 ? launch(decode_rope_kernel<DT, 1, 4, false, 1>, 4, false)                                         \
+                : launch(decode_rope_kernel<DT, 2, 4, false, 1>, 4, false))
+    int rc;
     if (levels) {
-        if (style == 0)
-            return s.dtype == RVQ_BF16 ? launch(decode_rope_kernel<RVQ_BF16, 1, false>)
-                                       : launch(decode_rope_kernel<RVQ_F16, 1, false>);
-        return s.dtype == RVQ_BF16 ? launch(decode_rope_kernel<RVQ_BF16, 2, false>)
-                                   : launch(decode_rope_kernel<RVQ_F16, 2, false>);
-    }
-    if (style == 0) {
-        switch (s.dtype) {
-        case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 1, true>);
-        case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 1, true>);
-        default: return launch(decode_rope_kernel<RVQ_F16, 1, true>);
+        if (s.dtype == RVQ_BF16) {
+            if ((rc = RVQ_ROPE_LEVELS(RVQ_BF16)) != RVQ_OK) return rc;
+            return RVQ_ROPE_F32(RVQ_BF16, 2);
         }
+        if ((rc = RVQ_ROPE_LEVELS(RVQ_F16)) != RVQ_OK) return rc;
+        return RVQ_ROPE_F32(RVQ_F16, 2);
     }
     switch (s.dtype) {
-    case RVQ_F32: return launch(decode_rope_kernel<RVQ_F32, 2, true>);
-    case RVQ_BF16: return launch(decode_rope_kernel<RVQ_BF16, 2, true>);
-    default: return launch(decode_rope_kernel<RVQ_F16, 2, true>);
+    case RVQ_F32: return RVQ_ROPE_F32(RVQ_F32, 0);
+    case RVQ_BF16: return RVQ_ROPE_F32(RVQ_BF16, 0);
+    default: return RVQ_ROPE_F32(RVQ_F16, 0);
     }
+#undef RVQ_ROPE_F32
+#undef RVQ_ROPE_LEVELS
 }
 
 int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
@@ -597,7 +657,8 @@ int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std1
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return RVQ_ERR_DEVICE;
     // which tables: see prepared.cuh
-    const bool both = decode_levels_supported(s) && s.K <= kDecodeWideK;      // decided on the device
+    const bool both = decode_levels_supported(s);                  // then the deviations decide on the device
+    const int lch = decode_slice_channels(s.K), fch = decode_exact_channels(s.K);
     const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
     auto launch = [&](auto kernel, int ch, bool f32t) -> int {
         const int ns = 32 / ch;
@@ -610,24 +671,28 @@ int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std1
         kernel<<<parts * ns, kDecThreads, smem, stream>>>(s, codes, std16, n, p + off, cb, out, stride, st);
         return check_launch();
     };
+#define RVQ_DEC_F32(DT, PICK)                                                                                       \
+    (fch == 4 ? launch(decode_sliced_kernel<DT, 4, true, PICK>, 4, true)                                           \
+              : launch(decode_sliced_kernel<DT, 2, true, PICK>, 2, true))
+#define RVQ_DEC_LEVELS(DT)                                                                                          \
+    (lch == 8 ? launch(decode_sliced_kernel<DT, 8, false, 1>, 8, false)                                            \
+              : launch(decode_sliced_kernel<DT, 4, false, 1>, 4, false))
+    int rc;
     if (both) {
-        int rc;
         if (s.dtype == RVQ_BF16) {
-            if ((rc = launch(decode_sliced_kernel<RVQ_BF16, 8, false, 1>, 8, false)) != RVQ_OK) return rc;
-            return launch(decode_sliced_kernel<RVQ_BF16, 4, true, 2>, 4, true);
+            if ((rc = RVQ_DEC_LEVELS(RVQ_BF16)) != RVQ_OK) return rc;
+            return RVQ_DEC_F32(RVQ_BF16, 2);
         }
-        if ((rc = launch(decode_sliced_kernel<RVQ_F16, 8, false, 1>, 8, false)) != RVQ_OK) return rc;
-        return launch(decode_sliced_kernel<RVQ_F16, 4, true, 2>, 4, true);
+        if ((rc = RVQ_DEC_LEVELS(RVQ_F16)) != RVQ_OK) return rc;
+        return RVQ_DEC_F32(RVQ_F16, 2);
     }
-    if (decode_exact_tables(s)) {
-        switch (s.dtype) {
-        case RVQ_F32: return launch(decode_sliced_kernel<RVQ_F32, 4, true, 0>, 4, true);
-        case RVQ_BF16: return launch(decode_sliced_kernel<RVQ_BF16, 4, true, 0>, 4, true);
-        default: return launch(decode_sliced_kernel<RVQ_F16, 4, true, 0>, 4, true);
-        }
+    switch (s.dtype) {
+    case RVQ_F32: return RVQ_DEC_F32(RVQ_F32, 0);
+    case RVQ_BF16: return RVQ_DEC_F32(RVQ_BF16, 0);
+    default: return RVQ_DEC_F32(RVQ_F16, 0);
     }
-    if (s.dtype == RVQ_BF16) return launch(decode_sliced_kernel<RVQ_BF16, 4, false, 0>, 4, false);
-    return launch(decode_sliced_kernel<RVQ_F16, 4, false, 0>, 4, false);
+#undef RVQ_DEC_F32
+#undef RVQ_DEC_LEVELS
 }
 
 }  // namespace rvq

@@ -41,16 +41,20 @@ constexpr int kDecodeWideK = 1536;                        // 128 bytes per code 
 constexpr int kDecodeMaxK = 3072;                         // 64 bytes per code per slice
 __host__ __device__ inline int decode_slice_channels(int K) { return K <= kDecodeWideK ? 8 : 4; }
 __host__ __device__ inline size_t decode_table_bytes(int K) { return (size_t)K * 512; }   // 32 channels x 8 stages x 2 bytes
-constexpr int kDecodeExactK = 1792;                       // float32 tables: 128 bytes per code per 4-channel slice
+constexpr int kDecodeExactWideK = 1792;                   // float32 tables: 128 bytes per code per 4-channel slice
+constexpr int kDecodeExactK = 3584;                       // ... 64 bytes per code per 2-channel slice
 // Which decoder serves a shape (group_dim 32, dim 128, depth <= 8; everything else gathers from global memory):
-//   - float32 table slices (exact sums, any output type) fit shared memory up to kDecodeExactK codes;
+//   - float32 table slices (exact sums, any output type) fit shared memory up to kDecodeExactK codes
+//     (4 channels per slice up to kDecodeExactWideK, 2 beyond);
 //   - 16-bit level tables (16-bit outputs only: their own rounding, 2^-9 or 2^-12 relative, dwarfs the
 //     tables') fit up to kDecodeMaxK codes and are the faster ones while the deviations are moderate;
-//   - up to kDecodeWideK codes and 16-bit outputs both fit, and the kernel chooses from the deviations.
+//   - where both fit (16-bit outputs, up to kDecodeMaxK codes) both kernels are launched and the one the
+//     deviations do not call for returns at once.
 __host__ __device__ inline bool decode_exact_tables(const Shape &s)
 {
     return s.gd == 32 && s.G == 4 && s.R <= 8 && s.K <= kDecodeExactK;
 }
+__host__ __device__ inline int decode_exact_channels(int K) { return K <= kDecodeExactWideK ? 4 : 2; }
 __host__ __device__ inline bool decode_levels_prepared(const Shape &s)    // the prepared block holds level tables
 {
     return s.gd == 32 && s.G == 4 && s.R <= 8 && s.K <= kDecodeMaxK;

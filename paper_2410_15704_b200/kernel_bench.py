@@ -78,6 +78,7 @@ def main():
     ap.add_argument("--iterations", type=int, default=10, help="Lloyd iterations per stage (kmeans)")
     ap.add_argument("--shape", default=None,
                     help="dim,group_dim,depth,codes[,layout] of the `ablation` workload, e.g. 128,32,6,1024")
+    ap.add_argument("--codes", type=int, default=None, help="codes per stage, for workloads that take a size")
     ap.add_argument("cases", nargs="+")
     ap.add_argument("--reps", type=int, default=10)
     args = ap.parse_args()
@@ -92,6 +93,8 @@ def main():
         elif spec.startswith("ablation") and args.shape:
             f = [int(t) for t in args.shape.split(",")]
             runs = [make(spec, dim=f[0], group_dim=f[1], depth=f[2], size=f[3], layout=f[4] if len(f) > 4 else 0)]
+        elif args.codes:
+            runs = [make(spec, size=args.codes)]
         else:
             runs = [make(spec)]
         for name, w in runs:

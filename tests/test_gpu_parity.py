@@ -82,6 +82,8 @@ def test_decode_bandwidth_full_size(layout):
     (2048, 16, rvq_synth.STRIDED, "f16"), (1537, 11, rvq_synth.CONTIGUOUS, "f16"),
     (3072, 12, rvq_synth.STRIDED, "bf16"), (1536, 11, rvq_synth.STRIDED, "bf16"),
     (3073, 12, rvq_synth.CONTIGUOUS, "bf16"),
+    (2048, 11, rvq_synth.CONTIGUOUS, "f32"), (2048, 16, rvq_synth.STRIDED, "f32"),      # float32 tables, 2-channel slices
+    (3584, 12, rvq_synth.STRIDED, "f16"), (3585, 12, rvq_synth.STRIDED, "f32"),
 ])
 def test_decode_large_codebooks(K, bits, layout, dtype):
     """More than 1536 codes per stage: narrow table slices (up to 3072 codes), gathers beyond."""

@@ -85,6 +85,9 @@ def test_decode_rope_level_tables(layout, pairing):
     run_case(128, 32, 8, 2048, 11, layout, "bf16", pairing, tokens=211)
     run_case(128, 32, 8, 3072, 12, layout, "f16", pairing, tokens=57)
     run_case(128, 32, 8, 2048, 16, layout, "bf16", pairing, tokens=57, std_scale=40.0)
+    # float32 tables with 2-channel slices: float32 outputs, and 16-bit outputs without a prepared block
+    run_case(128, 32, 8, 2048, 11, layout, "f32", pairing, tokens=57)
+    run_case(128, 32, 8, 3584, 12, layout, "bf16", pairing, tokens=57, with_prepared=False)
 
 
 def test_decode_rope_clamps_positions_and_rejects_bad_arguments():

@@ -164,8 +164,8 @@ int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n,
 /*
  * Decode (Section 2.2, last sentence; Section 3.2).  For every head vector and
  * channel c = channel(g, i): x_out[c] = std * sum_r C_r[code[g][r]][i], summed
- * in float32 and rounded once to x_dtype.  For dim 128 = 4 groups of 32 with
- * depth <= 8 the codebook entries are read from shared-memory tables: float32
+ * in float32 and rounded once to x_dtype.  For groups of 32 (a power-of-two number
+ * of them) with depth <= 8 the codebook entries are read from shared-memory tables: float32
  * copies (up to 3584 codes per stage) or, for 16-bit outputs and up to 3072
  * codes, 16-bit levels of each stage's value range kept in the prepared block.
  * With the levels the sum before the multiplication by std is within

@@ -162,13 +162,16 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
     const float exact_above = F32T ? INFINITY : (dp->err > 0.0f ? (ROPE != 0 ? 0.6e-3f : 0.9e-3f) / dp->err : INFINITY);
     __syncthreads();
 
-    const int64_t rows = n * 4;
+    // dim = 32 G with G a power of two; the stores of strided groups below are written for G = 4 (dim 128),
+    // other G store element by element
+    const int gs = __ffs(s.G) - 1;
+    const int64_t rows = n << gs;
     uint32_t bad = 0;
     for (int64_t row = (int64_t)part * kDecThreads + tid; row - tid < rows; row += (int64_t)parts * kDecThreads) {
         // (the loop bound keeps whole warps together for the shuffles below)
         const bool live = row < rows;
-        const int64_t v = live ? row >> 2 : 0;
-        const int g = (int)(row & 3);
+        const int64_t v = live ? row >> gs : 0;
+        const int g = (int)(row & (s.G - 1));
         // rotary decode: this row's cosines and sines, asked for first so that they arrive during the gather
         float2 rc[4];
         if (ROPE != 0) {
@@ -367,7 +370,14 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                 }
             }
         }
-        if constexpr (CH == 2) {
+        if (s.G != 4 && s.layout == RVQ_GROUP_STRIDED) {
+            // channel of place i: element * G + g
+            if (live) {
+#pragma unroll
+                for (int i = 0; i < CH; ++i)
+                    store_from_float(out, v * stride + (int64_t)slice_element<CH, ROPE>(s.layout, slice, i) * s.G + g, DT, o8[i]);
+            }
+        } else if constexpr (CH == 2) {
             // two places per thread
             if (DT == RVQ_F32) {
                 float *o = reinterpret_cast<float *>(out) + v * stride;
@@ -584,7 +594,7 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     for (int b = 0; b < 31; ++b)
         if (per_position == (1 << b)) shift = b;
     RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions, shift};
-    const bool f32t = decode_exact_tables(s);
+    const bool f32t = decode_exact_tables(s) && s.G == 4;         // the lane exchanges of the rotation are written for 4 groups
     const bool levels = prepared != nullptr && decode_levels_supported(s) && decode_slice_channels(s.K) == 4;
     if (!f32t || n > 0x7FFFFFFF) {
         const int per_vec = s.G * (s.gd / 4);
@@ -604,7 +614,7 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     const uint8_t *dsec = nullptr;
     if (levels)
         dsec = reinterpret_cast<const uint8_t *>(prepared) + (kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256;
-    const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
+    const int64_t tiles = (n * s.G + kDecThreads - 1) / kDecThreads;
     auto launch = [&](auto kernel, int ch, bool f32_tables) -> int {
         const int ns = 32 / ch;
         const size_t smem = (size_t)s.K * (f32_tables ? 32 : 16) * ch;
@@ -659,7 +669,7 @@ int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std1
     // which tables: see prepared.cuh
     const bool both = decode_levels_supported(s);                  // then the deviations decide on the device
     const int lch = decode_slice_channels(s.K), fch = decode_exact_channels(s.K);
-    const int64_t tiles = (n * 4 + kDecThreads - 1) / kDecThreads;
+    const int64_t tiles = (n * s.G + kDecThreads - 1) / kDecThreads;
     auto launch = [&](auto kernel, int ch, bool f32t) -> int {
         const int ns = 32 / ch;
         const size_t smem = (size_t)s.K * (f32t ? 32 : 16) * ch;

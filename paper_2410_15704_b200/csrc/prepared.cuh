@@ -43,7 +43,8 @@ __host__ __device__ inline int decode_slice_channels(int K) { return K <= kDecod
 __host__ __device__ inline size_t decode_table_bytes(int K) { return (size_t)K * 512; }   // 32 channels x 8 stages x 2 bytes
 constexpr int kDecodeExactWideK = 1792;                   // float32 tables: 128 bytes per code per 4-channel slice
 constexpr int kDecodeExactK = 3584;                       // ... 64 bytes per code per 2-channel slice
-// Which decoder serves a shape (group_dim 32, dim 128, depth <= 8; everything else gathers from global memory):
+// Which decoder serves a shape (group_dim 32, a power-of-two number of groups up to 32, depth <= 8; everything
+// else gathers from global memory):
 //   - float32 table slices (exact sums, any output type) fit shared memory up to kDecodeExactK codes
 //     (4 channels per slice up to kDecodeExactWideK, 2 beyond);
 //   - 16-bit level tables (16-bit outputs only: their own rounding, 2^-9 or 2^-12 relative, dwarfs the
@@ -52,12 +53,12 @@ constexpr int kDecodeExactK = 3584;                       // ... 64 bytes per co
 //     deviations do not call for returns at once.
 __host__ __device__ inline bool decode_exact_tables(const Shape &s)
 {
-    return s.gd == 32 && s.G == 4 && s.R <= 8 && s.K <= kDecodeExactK;
+    return s.gd == 32 && s.G <= 32 && (s.G & (s.G - 1)) == 0 && s.R <= 8 && s.K <= kDecodeExactK;
 }
 __host__ __device__ inline int decode_exact_channels(int K) { return K <= kDecodeExactWideK ? 4 : 2; }
 __host__ __device__ inline bool decode_levels_prepared(const Shape &s)    // the prepared block holds level tables
 {
-    return s.gd == 32 && s.G == 4 && s.R <= 8 && s.K <= kDecodeMaxK;
+    return s.gd == 32 && s.G <= 32 && (s.G & (s.G - 1)) == 0 && s.R <= 8 && s.K <= kDecodeMaxK;
 }
 __host__ __device__ inline bool decode_levels_supported(const Shape &s)
 {

@@ -115,6 +115,26 @@ def test_decode_large_deviations_take_the_exact_route(K, layout, every):
     assert_recon_match(got, w.codes, std_bits, w.codebooks, w.dim, layout, cfg.x_dtype)
 
 
+@pytest.mark.parametrize("dim,K,bits,layout,dtype,std_scale", [
+    (256, 1024, 10, rvq_synth.CONTIGUOUS, "bf16", 1.0), (256, 1024, 16, rvq_synth.STRIDED, "bf16", 1.0),
+    (256, 2048, 11, rvq_synth.STRIDED, "f16", 1.0), (256, 2048, 11, rvq_synth.CONTIGUOUS, "f32", 1.0),
+    (256, 1024, 16, rvq_synth.STRIDED, "bf16", 50.0), (64, 512, 9, rvq_synth.STRIDED, "bf16", 1.0),
+    (512, 300, 9, rvq_synth.CONTIGUOUS, "f16", 1.0),
+])
+def test_decode_other_head_sizes(dim, K, bits, layout, dtype, std_scale):
+    """Head vectors of 2, 8 and 16 groups of 32 (head_dim 64, 256, 512) on the table kernels."""
+    g = np.random.default_rng(dim + K + layout)
+    n, G, R = 1531, dim // 32, 8
+    codes = g.integers(0, K, size=(n, G, R)).astype(np.int32)
+    std_bits = (std_scale * (np.abs(1.0 + 0.25 * g.normal(size=n)) + 0.05)).astype(np.float16).view(np.uint16)
+    cb = np.stack([g.normal(scale=0.5 * 0.75 ** r, size=(K, 32)) for r in range(R)]).astype(np.float32)
+    cfg = rvq.make_config(dim, 32, layout, R, K, bits, DT[dtype], 0)
+    got, st = gpu_decode(cfg, codes, std_bits, cb, n, row_stride=dim + 8)
+    assert np.all(got[:, dim:] == 7.0)
+    assert_recon_match(got, codes, std_bits, cb, dim, layout, cfg.x_dtype)
+    assert st["bad_codes"] == 0
+
+
 def test_decode_head_major_tiles():
     """Output rows written through a row stride: [head][token][dim] tiles."""
     w = rvq_synth.decode_bandwidth(tokens=1024)

@@ -1,8 +1,9 @@
-// Bandwidth decode for dim 128 = 4 groups of 32, depth <= 8 (Section 2.2, last
+// Bandwidth decode for groups of 32 (a power-of-two number of them per head
+// vector; written around dim 128 = 4 groups), depth <= 8 (Section 2.2, last
 // sentence; Section 3.2).
 //
 // Every output element needs one codeword element per stage, so a head vector of
-// 256 output bytes gathers 1024 table entries: the gather, not HBM, is the
+// 128 channels (256 output bytes) gathers 1024 table entries: the gather, not HBM, is the
 // limit, and it has to come from shared memory without bank conflicts.
 //   - A CTA keeps one channel slice (CH = 8 of the 32 codeword channels, 4 when
 //     there are more than 1536 codes per stage) of all stages as 16-bit levels:

@@ -196,7 +196,7 @@ int rvq_decode(const rvq_config *cfg /* host */, const void *codes, const uint16
  *   cos_sin               in  device float32 [positions][dim/2][2], 16-byte aligned, e.g. from
  *                             rvq_rope_table
  *   prepared              in  block of rvq_prepare_codebooks for these codebooks, or NULL
- * dim 128 in 4 groups of 32 with depth <= 8: up to 3584 codes per stage float32
+ * Two or more groups of 32 (a power-of-two number) with depth <= 8: up to 3584 codes per stage float32
  * shared-memory tables (exact float32 sums); with 16-bit outputs, a prepared block and
  * 1537..3072 codes also the level tables described under rvq_decode, chosen when the
  * deviations are moderate (a head vector whose std would make std * err exceed 0.6e-3

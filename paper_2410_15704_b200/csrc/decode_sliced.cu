@@ -181,31 +181,32 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
             const uint32_t token = ra.shift >= 0 ? (uint32_t)v >> ra.shift : (uint32_t)v / (uint32_t)ra.per_position;
             int pos = live ? __ldg(ra.position + token) : 0;
             pos = min(max(pos, 0), ra.positions - 1);
-            const float2 *cs = ra.table + (size_t)pos * 64;
+            const int hG = s.G >> 1;                                  // groups per half of the head vector
+            const float2 *cs = ra.table + (size_t)pos * (16 * s.G);      // dim / 2 pairs per position
             if (CH == 2) {
                 // one pair in the thread (half-split pairs on strided groups: pair 4 slice + g; adjacent pairs on
                 // contiguous groups: pair 16 g + slice), or two places whose partners sit in another lane
-                if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) rc[0] = __ldg(cs + slice * 4 + g);
+                if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) rc[0] = __ldg(cs + slice * s.G + g);
                 else if (ROPE == 2 && s.layout != RVQ_GROUP_STRIDED) rc[0] = __ldg(cs + g * 16 + slice);
-                else if (ROPE == 1) {                                  // pairs 32 (g & 1) + 2 slice + i
-                    const float4 cc = __ldg(reinterpret_cast<const float4 *>(cs + (g & 1) * 32 + slice * 2));
+                else if (ROPE == 1) {                                  // pairs 32 (g mod G/2) + 2 slice + i
+                    const float4 cc = __ldg(reinterpret_cast<const float4 *>(cs + (g & (hG - 1)) * 32 + slice * 2));
                     rc[0] = make_float2(cc.x, cc.y); rc[1] = make_float2(cc.z, cc.w);
-                } else {                                               // pairs 2 (2 slice + i) + g / 2
-                    rc[0] = __ldg(cs + slice * 4 + (g >> 1)); rc[1] = __ldg(cs + slice * 4 + 2 + (g >> 1));
+                } else {                                               // pairs (G / 2) (2 slice + i) + g / 2
+                    rc[0] = __ldg(cs + (slice * 2) * hG + (g >> 1)); rc[1] = __ldg(cs + (slice * 2 + 1) * hG + (g >> 1));
                 }
-            } else if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) {   // pairs 4 (2 slice + i) + g
-                rc[0] = __ldg(cs + slice * 8 + g); rc[1] = __ldg(cs + slice * 8 + 4 + g);
+            } else if (ROPE == 1 && s.layout == RVQ_GROUP_STRIDED) {   // pairs G (2 slice + i) + g
+                rc[0] = __ldg(cs + (slice * 2) * s.G + g); rc[1] = __ldg(cs + (slice * 2 + 1) * s.G + g);
             } else if (ROPE == 2 && s.layout != RVQ_GROUP_STRIDED) {   // pairs 16 g + 2 slice + i
                 const float4 cc = __ldg(reinterpret_cast<const float4 *>(cs + g * 16 + slice * 2));
                 rc[0] = make_float2(cc.x, cc.y); rc[1] = make_float2(cc.z, cc.w);
-            } else if (ROPE == 1) {                                    // pairs 32 (g & 1) + 4 slice + i
-                const float4 *q = reinterpret_cast<const float4 *>(cs + (g & 1) * 32 + slice * 4);
+            } else if (ROPE == 1) {                                    // pairs 32 (g mod G/2) + 4 slice + i
+                const float4 *q = reinterpret_cast<const float4 *>(cs + (g & (hG - 1)) * 32 + slice * 4);
                 const float4 lo = __ldg(q), hi = __ldg(q + 1);
                 rc[0] = make_float2(lo.x, lo.y); rc[1] = make_float2(lo.z, lo.w);
                 rc[2] = make_float2(hi.x, hi.y); rc[3] = make_float2(hi.z, hi.w);
             } else {                                                   // pairs 2 (4 slice + i) + g / 2
 #pragma unroll
-                for (int i = 0; i < 4; ++i) rc[i] = __ldg(cs + (slice * 4 + i) * 2 + (g >> 1));
+                for (int i = 0; i < 4; ++i) rc[i] = __ldg(cs + (slice * 4 + i) * hG + (g >> 1));
             }
         }
         // the 8 codes of this row as 4 words, stage r in half r
@@ -359,10 +360,10 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
                     o8[2 * i + 1] = b * rc[i].x + a * rc[i].y;
                 }
             } else {
-                // the partner is the same place of another group: lane g ^ 2 (half-split pairs, contiguous
-                // groups: channels 32 g + e and 32 (g ^ 2) + e) or lane g ^ 1 (adjacent pairs, strided groups:
-                // channels 4 e + g and 4 e + (g ^ 1))
-                const int other = ROPE == 1 ? 2 : 1;
+                // the partner is the same place of another group: lane g ^ G/2 (half-split pairs, contiguous
+                // groups: channels 32 g + e and 32 (g ^ G/2) + e) or lane g ^ 1 (adjacent pairs, strided groups:
+                // channels G e + g and G e + (g ^ 1))
+                const int other = ROPE == 1 ? (s.G >> 1) : 1;
                 const bool first = (g & other) == 0;
 #pragma unroll
                 for (int i = 0; i < CH; ++i) {
@@ -595,7 +596,7 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     for (int b = 0; b < 31; ++b)
         if (per_position == (1 << b)) shift = b;
     RopeArgs ra{position, per_position, reinterpret_cast<const float2 *>(table), positions, shift};
-    const bool f32t = decode_exact_tables(s) && s.G == 4;         // the lane exchanges of the rotation are written for 4 groups
+    const bool f32t = decode_exact_tables(s) && s.G >= 2;         // (one group: the pairs are inside a row; gather kernel)
     const bool levels = prepared != nullptr && decode_levels_supported(s) && decode_slice_channels(s.K) == 4;
     if (!f32t || n > 0x7FFFFFFF) {
         const int per_vec = s.G * (s.gd / 4);

@@ -72,6 +72,13 @@ def test_decode_rope_table_path(layout, pairing, dtype):
     (128, 32, 6, 1024, 10, rvq_synth.CONTIGUOUS, "f16", rvq.ROPE_ADJACENT),   # packed codes on the table path
     (256, 32, 4, 512, 16, rvq_synth.STRIDED, "bf16", rvq.ROPE_HALVES),
     (64, 16, 8, 64, 6, rvq_synth.CONTIGUOUS, "f32", rvq.ROPE_ADJACENT),
+    (256, 32, 8, 1024, 10, rvq_synth.CONTIGUOUS, "bf16", rvq.ROPE_HALVES),    # head_dim 256 on the table kernels
+    (256, 32, 8, 1024, 16, rvq_synth.CONTIGUOUS, "f16", rvq.ROPE_ADJACENT),
+    (256, 32, 8, 2048, 11, rvq_synth.STRIDED, "bf16", rvq.ROPE_ADJACENT),
+    (256, 32, 8, 2048, 11, rvq_synth.STRIDED, "f32", rvq.ROPE_HALVES),
+    (64, 32, 8, 512, 9, rvq_synth.STRIDED, "bf16", rvq.ROPE_HALVES),          # two groups
+    (64, 32, 8, 512, 9, rvq_synth.CONTIGUOUS, "bf16", rvq.ROPE_HALVES),
+    (32, 32, 4, 256, 8, rvq_synth.CONTIGUOUS, "bf16", rvq.ROPE_HALVES),       # one group: gather kernel
 ])
 def test_decode_rope_other_shapes(dim, gd, R, K, bits, layout, dtype, pairing):
     run_case(dim, gd, R, K, bits, layout, dtype, pairing, tokens=97, heads=4, max_pos=5000)

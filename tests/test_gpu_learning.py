@@ -68,23 +68,23 @@ def residual_energy(x, cbs, layout):
     return float((enc["residual"] ** 2).mean())
 
 
-def clustered_vectors(seed, n, K, layout):
-    """Head vectors whose four groups each sit near one of K well-separated centres."""
+def clustered_vectors(seed, n, K, layout, G=4):
+    """Head vectors whose G groups each sit near one of K well-separated centres."""
     g = np.random.default_rng(seed)
     centres = g.normal(size=(K, 32)) * 3.0
-    labels = g.integers(0, K, size=(n, 4))
-    rows = centres[labels] + 0.05 * g.normal(size=(n, 4, 32))            # [n][G][32]
-    x = rows.reshape(n, 128) if layout == rvq_synth.CONTIGUOUS else rows.transpose(0, 2, 1).reshape(n, 128)
+    labels = g.integers(0, K, size=(n, G))
+    rows = centres[labels] + 0.05 * g.normal(size=(n, G, 32))            # [n][G][32]
+    x = rows.reshape(n, 32 * G) if layout == rvq_synth.CONTIGUOUS else rows.transpose(0, 2, 1).reshape(n, 32 * G)
     x = torch.from_numpy(x).to(torch.bfloat16).float().numpy()           # exactly representable
     return x, labels.reshape(-1)
 
 
-@pytest.mark.parametrize("layout", [rvq_synth.CONTIGUOUS, rvq_synth.STRIDED])
-def test_kmeans_init_on_separated_clusters(layout):
-    n, K, R, iters = 1500, 16, 3, 4                                      # 6000 rows: ragged last tile
-    x, labels = clustered_vectors(31, n, K, layout)
+@pytest.mark.parametrize("layout,G", [(rvq_synth.CONTIGUOUS, 4), (rvq_synth.STRIDED, 4), (rvq_synth.STRIDED, 8)])
+def test_kmeans_init_on_separated_clusters(layout, G):
+    n, K, R, iters = 1500, 16, 3, 4                                      # ragged last tile
+    x, labels = clustered_vectors(31, n, K, layout, G)
     seeds = np.stack([np.array([np.flatnonzero(labels == k)[r] for k in range(K)]) for r in range(R)]).astype(np.int64)
-    cfg = rvq.make_config(128, 32, layout, R, K, 16, rvq.BF16, 0)
+    cfg = rvq.make_config(32 * G, 32, layout, R, K, 16, rvq.BF16, 0)
     got, _, _ = gpu_kmeans(cfg, x, n, seeds, iters)
     ref = oracle.kmeans_init(x, seeds, iters, 32, layout)
     # stage 0: every row sits far inside its cluster, so the assignments cannot differ

@@ -155,6 +155,12 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&u)[32])
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : RVQ_INOUT32(u) : : "memory");
 }
+__device__ __forceinline__ void tmem_ld_wait3(uint32_t (&u)[32], uint32_t (&v)[32], uint32_t (&w)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : RVQ_INOUT32(u) : : "memory");
+    asm volatile("" : RVQ_INOUT32(v) : : "memory");
+    asm volatile("" : RVQ_INOUT32(w) : : "memory");
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&u)[32])
 {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -166,18 +172,34 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&u)[32
 
 // Per-row state of one stage's sweep over the scores.
 struct Sweep {
-    float m1, thr, win;      // running minimum of the block minima, m1 + win, error window
+    float m1, thr, win;      // running minimum of the block minima, threshold(m1), error window
+    float zz;                // squared norm of the scaled residual: m1 + zz is the best squared distance
     int cnt;                 // listed blocks (kListCap + 1: the list overflowed)
     float d[11];             // minimum per cell position (3 columns each, the last one 2)
+    float k[3];              // minimum per column position inside its cell
 };
 
-// Minima of the eleven 3-column cells of a 32-column block, and the block minimum.
-__device__ __forceinline__ float block_cells(const uint32_t (&u)[32], float (&t)[11])
+// One 32-column block of scores: folds its eleven 3-column cell minima into w.d and the minima of
+// the three in-cell column positions into w.k; returns the block minimum.  A column that could be
+// the argmin is thereby pinned to (listed block) x (cell position) x (position in the cell).
+__device__ __forceinline__ float fold_block(Sweep &w, const uint32_t (&u)[32])
 {
+    float t[11];
 #pragma unroll
     for (int q = 0; q < 10; ++q)
         t[q] = min3(__uint_as_float(u[3 * q]), __uint_as_float(u[3 * q + 1]), __uint_as_float(u[3 * q + 2]));
     t[10] = fminf(__uint_as_float(u[30]), __uint_as_float(u[31]));
+#pragma unroll
+    for (int q = 0; q < 11; ++q) w.d[q] = fminf(w.d[q], t[q]);
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        float m = w.k[c];
+#pragma unroll
+        for (int q = 0; q < 10; q += 2)
+            m = min3(m, __uint_as_float(u[3 * q + c]), __uint_as_float(u[3 * q + 3 + c]));
+        if (c < 2) m = fminf(m, __uint_as_float(u[30 + c]));      // the last cell has two columns
+        w.k[c] = m;
+    }
     return min3(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])), t[9], t[10]);
 }
 
@@ -185,12 +207,21 @@ __device__ __forceinline__ float block_cells(const uint32_t (&u)[32], float (&t)
 // Branch-free: the value is always written to the next free slot and the slot
 // is claimed only when it belongs on the list; slot kListCap is scratch once
 // the list has overflowed.
+// A column can only be the exact-L2 choice (in real arithmetic, and in the float32 direct-form
+// arithmetic of the all-float32 kernel, whose relative error on a distance is below 34 * 2^-24) if its
+// approximate score is at most threshold(m1): the window covers the approximation error of both
+// scores, the last term the float32 evaluation error of both distances (2 * 34 * 2^-24 < 2^-17.5).
+__device__ __forceinline__ float threshold(const Sweep &w, float m1)
+{
+    return m1 + w.win + 5.4e-6f * (fmaxf(m1 + w.zz, 0.0f) + w.win);
+}
+
 __device__ __forceinline__ void list_block(Sweep &w, float cb_min, int block, float *list_v, uint16_t *list_i,
                                            int stride)
 {
     const bool app = cb_min <= w.thr;
     w.m1 = fminf(w.m1, cb_min);
-    w.thr = w.m1 + w.win;
+    w.thr = threshold(w, w.m1);
     if (app && w.cnt == kListCap) {
         // full: drop entries that left the window as the minimum came down
         int keep = 0;
@@ -299,6 +330,12 @@ encode_tensor_kernel(const Params p)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_word;
+
+    // The four role warps run one lane each and need few registers; their share goes to the
+    // epilogue warps, which hold three 32-column blocks of scores at a time
+    // (12 warps x 32 x 152 + 4 warps x 32 x 40 = 63488 of the 65536 the block was launched with).
+    if (warp >= kEpiThreads / 32) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    else asm volatile("setmaxnreg.inc.sync.aligned.u32 152;");
 
     if (warp == kEpiThreads / 32 + kTiles) {
         // ------------------------------------------------------------ operand loader
@@ -482,55 +519,51 @@ encode_tensor_kernel(const Params p)
                 for (int i = 0; i < 32; ++i) z_park[i * kRowsPerPass] = z[i];
                 Sweep w;
                 w.win = 2.125f * (prm.a * sqrtf(zz) * 1.0001f + prm.b);    // 2 * bound, with slack for this arithmetic
+                w.zz = zz;
                 w.m1 = INFINITY; w.thr = INFINITY; w.cnt = 0;
 #pragma unroll
                 for (int q = 0; q < 11; ++q) w.d[q] = INFINITY;
+                w.k[0] = w.k[1] = w.k[2] = INFINITY;
                 const bool force_scan = !(zmax < 60000.0f) || !(w.win < INFINITY);
 
 #pragma unroll 1
                 for (int c = 0; c < S && ok; ++c) {
                     if (c == S - 1 && w.cnt > 0) {
                         // Before the last chunk the running winner is the final one most of the time:
-                        // start fetching its cell's three codewords while the MMA chain runs.
-                        int pb = 0, pq = 0;
+                        // start fetching its codeword while the MMA chain runs.
+                        int pb = 0, pq = 0, pk = 0;
 #pragma unroll
                         for (int e = kListCap - 1; e >= 0; --e)
                             if (e < w.cnt && list_v[e * kRowsPerPass] == w.m1) pb = list_i[e * kRowsPerPass];
 #pragma unroll
                         for (int q = 10; q >= 0; --q)
                             if (w.d[q] == w.m1) pq = q;
-                        const int pj = min(pb * 32 + 3 * pq, s.K - 1);
-                        const float *pp = cbr + (size_t)pj * 32;
-                        asm volatile("prefetch.global.L1 [%0];" ::"l"(pp));
-                        asm volatile("prefetch.global.L1 [%0];" ::"l"(pp + 32));
-                        asm volatile("prefetch.global.L1 [%0];" ::"l"(pp + 64));
+                        if (w.k[1] == w.m1) pk = 1;
+                        if (w.k[2] == w.m1) pk = 2;
+                        const int pj = min(pb * 32 + 3 * pq + pk, s.K - 1);
+                        asm volatile("prefetch.global.L1 [%0];" ::"l"(cbr + (size_t)pj * 32));
                     }
                     ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag);
                     ok = __all_sync(0xFFFFFFFFu, ok);          // tcgen05.ld below needs the whole warp
                     ++chunk_use;
                     if (!ok) break;
                     tc_fence_after();
-                    // Four 32-column blocks.  Only the cell minima of a block are taken between two
-                    // loads, so that the accumulator is handed back to the MMA issuer as early as
-                    // possible; the rest of the reduction runs while the next chain computes.
-                    uint32_t ua[32], ub[32];
-                    float t0[11], t1[11], t2[11], t3[11];
+                    // Four 32-column blocks, three of them in flight at once; the fourth is asked for as
+                    // soon as the first has been reduced, and the accumulator goes back to the MMA issuer
+                    // when it has landed.
+                    uint32_t ua[32], ub[32], uc[32];
                     tmem_ld32_issue(taddr, ua);
-                    tmem_ld_wait(ua);
                     tmem_ld32_issue(taddr + 32, ub);
-                    const float c0 = block_cells(ua, t0);
-                    tmem_ld_wait(ub);
-                    tmem_ld32_issue(taddr + 64, ua);
-                    const float c1 = block_cells(ub, t1);
+                    tmem_ld32_issue(taddr + 64, uc);
+                    tmem_ld_wait3(ua, ub, uc);
+                    const float c0 = fold_block(w, ua);
+                    tmem_ld32_issue(taddr + 96, ua);
+                    const float c1 = fold_block(w, ub);
+                    const float c2 = fold_block(w, uc);
                     tmem_ld_wait(ua);
-                    tmem_ld32_issue(taddr + 96, ub);
-                    const float c2 = block_cells(ua, t2);
-                    tmem_ld_wait(ub);
                     tc_fence_before();
                     mbar_arrive(BAR(kBarAccFree + tile));        // the accumulator may be overwritten
-                    const float c3 = block_cells(ub, t3);
-#pragma unroll
-                    for (int q = 0; q < 11; ++q) w.d[q] = min3(min3(w.d[q], t0[q], t1[q]), t2[q], t3[q]);
+                    const float c3 = fold_block(w, ua);
                     list_block(w, c0, c * 4, list_v, list_i, kRowsPerPass);
                     list_block(w, c1, c * 4 + 1, list_v, list_i, kRowsPerPass);
                     list_block(w, c2, c * 4 + 2, list_v, list_i, kRowsPerPass);
@@ -542,16 +575,12 @@ encode_tensor_kernel(const Params p)
                 for (int i = 0; i < 32; ++i) z[i] = z_park[i * kRowsPerPass];
                 const float m1 = w.m1;
                 const int cnt = w.cnt;
-                float d[11];
-#pragma unroll
-                for (int q = 0; q < 11; ++q) d[q] = w.d[q];
-                const float win = w.win;
-                if (!ok) break;
 
-                // ---- stage end: exact choice among the columns that can still be the argmin.
-                // Common case (one listed block, one cell position): its three columns are
-                // re-scored by the row's own thread, all lanes in step.
-                const float lim = m1 + win;
+                // ---- stage end: the columns that can still be the exact argmin are those of a listed
+                // block, at a listed cell position, at a listed place inside the cell.  When each of the
+                // three lists has one entry (almost always) that column is the choice: every other
+                // column is farther than the approximation and float32 evaluation errors can bridge.
+                const float lim = threshold(w, m1);
                 int b1 = 0, nlisted = 0;
                 {
                     bool found = false;
@@ -564,42 +593,28 @@ encode_tensor_kernel(const Params p)
                         if (live && !found && fv == m1) { found = true; b1 = fi; }
                     }
                 }
-                int q1 = 0, ncells = 0;
+                uint32_t qmask = 0u, kmask = 0u;
+                int q1 = 0, k1 = 0;
 #pragma unroll
                 for (int q = 10; q >= 0; --q) {
-                    if (d[q] <= lim) ++ncells;
-                    if (d[q] == m1) q1 = q;
+                    if (w.d[q] <= lim) qmask |= 1u << q;
+                    if (w.d[q] == m1) q1 = q;
                 }
-                int bj = 0;
-                float best = INFINITY;
-                {
-                    // the three columns of the cell, scored together so that their loads overlap
-                    const int j0 = b1 * 32 + 3 * q1;
-                    const bool in1 = 3 * q1 + 1 < 32 && j0 + 1 < s.K, in2 = 3 * q1 + 2 < 32 && j0 + 2 < s.K;
-                    const float *e0 = cbr + (size_t)(j0 < s.K ? j0 : 0) * 32;
-                    const float *e1 = in1 ? e0 + 32 : e0, *e2 = in2 ? e0 + 64 : e0;
-                    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f;
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float u0[8], u1[8], u2[8];
-                        ldg256(e0 + 8 * q, u0); ldg256(e1 + 8 * q, u1); ldg256(e2 + 8 * q, u2);
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            float t;
-                            t = z[8 * q + k] - u0[k]; a0 = fmaf(t, t, a0);
-                            t = z[8 * q + k] - u1[k]; a1 = fmaf(t, t, a1);
-                            t = z[8 * q + k] - u2[k]; a2 = fmaf(t, t, a2);
-                        }
-                    }
-                    if (j0 < s.K) { best = a0; bj = j0; }
-                    if (in1 && a1 < best) { best = a1; bj = j0 + 1; }
-                    if (in2 && a2 < best) { best = a2; bj = j0 + 2; }
+                for (int c = 2; c >= 0; --c) {
+                    if (w.k[c] <= lim) kmask |= 1u << c;
+                    if (w.k[c] == m1) k1 = c;
                 }
-                const bool scan_all = force_scan || cnt == 0 || cnt > kListCap;
-                const bool flagged = !deg && (scan_all || nlisted * ncells > 1);
-                // Rows with more than one candidate: the whole warp re-scores every column of
-                // every listed block of one such row at a time (or all columns when the list
-                // overflowed), then reduces to the smallest distance, lowest index on ties.
+                const int j1 = b1 * 32 + 3 * q1 + k1;
+                // (a padded column scores 60000: if nothing real scored less, scan everything)
+                const bool scan_all = force_scan || cnt == 0 || cnt > kListCap || !(m1 < 59000.0f);
+                const bool unique = nlisted == 1 && (qmask & (qmask - 1u)) == 0u && (kmask & (kmask - 1u)) == 0u && j1 < s.K;
+                const bool flagged = !deg && (scan_all || !unique);
+                int bj = j1 < s.K ? j1 : 0;
+                // Rows with more than one candidate: the whole warp re-scores the candidate columns of
+                // every listed block of one such row at a time (lane = place in the block; all columns
+                // when the list overflowed) exactly in float32, direct form, then reduces to the
+                // smallest distance, lowest index on ties.
                 uint32_t todo = __ballot_sync(0xFFFFFFFFu, flagged);
                 while (todo) {
                     const int src = __ffs(todo) - 1;
@@ -609,8 +624,12 @@ encode_tensor_kernel(const Params p)
                     for (int i = 0; i < 32; ++i) zs[i] = z_park[i * kRowsPerPass + (src - lane)];
                     const float lim_s = __shfl_sync(0xFFFFFFFFu, lim, src);
                     const int cnt_s = __shfl_sync(0xFFFFFFFFu, cnt, src);
+                    const uint32_t qmask_s = __shfl_sync(0xFFFFFFFFu, qmask, src);
+                    const uint32_t kmask_s = __shfl_sync(0xFFFFFFFFu, kmask, src);
                     const bool all_s = __shfl_sync(0xFFFFFFFFu, (int)scan_all, src) != 0;
                     const int row_s = rloc - lane + src;
+                    const int lq = lane >= 30 ? 10 : lane / 3;
+                    const bool mine = ((qmask_s >> lq) & 1u) && ((kmask_s >> (lane - 3 * lq)) & 1u);
                     float bv = INFINITY;
                     int bi = 0x7FFFFFFF;
                     if (all_s) {
@@ -623,8 +642,10 @@ encode_tensor_kernel(const Params p)
                             const float fv = reinterpret_cast<const float *>(smem + kOffListV)[e * kRowsPerPass + row_s];
                             if (!(fv <= lim_s)) continue;                              // warp-uniform
                             const int j = (int)reinterpret_cast<const uint16_t *>(smem + kOffListI)[e * kRowsPerPass + row_s] * 32 + lane;
-                            const float dj = exact_distance(zs, cbr + (size_t)(j < s.K ? j : 0) * 32);
-                            if (j < s.K && dj < bv) { bv = dj; bi = j; }
+                            if (mine && j < s.K) {
+                                const float dj = exact_distance(zs, cbr + (size_t)j * 32);
+                                if (dj < bv) { bv = dj; bi = j; }
+                            }
                         }
                     }
 #pragma unroll
@@ -634,7 +655,7 @@ encode_tensor_kernel(const Params p)
                         if (ov < bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
                     }
                     if (lane == src) {
-                        bj = bi; best = bv;
+                        bj = bi < s.K ? bi : 0;
                         if (all_s) ++n_exhaustive; else ++n_rescored;
                     }
                 }

@@ -237,6 +237,38 @@ def test_check_codes_flags_planted_errors():
     assert st[3, 2, 0] == 0
 
 
+def test_check_codes_verdicts_on_hand_built_near_ties():
+    """Every verdict of the checker (exact, near tie inside / outside the window, third-best
+    inside the window, tie broken upward, out of range, the denominator of the relative gap,
+    conditioning of stage 1 on the given stage-0 code) against cases worked by hand."""
+    x = np.array([[2.0, -2.0, 2.0, -2.0]])
+    z = np.array([1.0, -1.0, 1.0, -1.0])
+    stage1 = np.array([[-0.9, 0, 0, 0], [0, -0.9, 0, 0], [0, 0, 5.0, 0]])
+    cases = 0
+    with open(os.path.join(GOLDEN, "check_codes_near_tie.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            name, tol, d0, d1, d2, axes, given, status, gap = line.split()
+            stage0 = np.tile(z, (3, 1))
+            for j, (dj, ax) in enumerate(zip((d0, d1, d2), axes.split(","))):
+                stage0[j, int(ax)] += math.sqrt(float(dj))
+            given = [int(t) for t in given.split(",")]
+            want = [int(t) for t in status.split(",")]
+            cb = np.stack([stage0, stage1])[: len(given)]
+            codes = np.array(given, dtype=np.int32).reshape(1, 1, len(given))
+            st, wrong, g = oracle.check_codes(x, codes, cb, 0, tol=float(tol), want_gap=True)
+            assert st.reshape(-1).tolist() == want, name
+            assert wrong == sum(1 for t in want if t >= 2), name
+            want_gap = float(Fraction(gap)) if "/" in gap else float(gap)
+            if math.isinf(want_gap):
+                assert math.isinf(g[0, 0, 0]), name
+            else:
+                assert abs(g[0, 0, 0] - want_gap) <= 1e-9, (name, g[0, 0, 0])
+            cases += 1
+    assert cases == 9
+
+
 # ---------------------------------------------------------------- number formats
 
 def test_f16_matches_numpy():

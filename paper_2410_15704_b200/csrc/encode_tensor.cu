@@ -155,11 +155,12 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&u)[32])
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : RVQ_INOUT32(u) : : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait3(uint32_t (&u)[32], uint32_t (&v)[32], uint32_t (&w)[32])
+__device__ __forceinline__ void tmem_ld_wait4(uint32_t (&u)[32], uint32_t (&v)[32], uint32_t (&w)[32], uint32_t (&x)[32])
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : RVQ_INOUT32(u) : : "memory");
     asm volatile("" : RVQ_INOUT32(v) : : "memory");
     asm volatile("" : RVQ_INOUT32(w) : : "memory");
+    asm volatile("" : RVQ_INOUT32(x) : : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&u)[32])
 {
@@ -174,15 +175,17 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&u)[32
 struct Sweep {
     float m1, thr, win;      // running minimum of the block minima, threshold(m1), error window
     float zz;                // squared norm of the scaled residual: m1 + zz is the best squared distance
-    int cnt;                 // listed blocks (kListCap + 1: the list overflowed)
+    int cnt;                 // listed chunks (kListCap + 1: the list overflowed)
+    float bb[4];             // minimum per 32-column block position inside its 128-column chunk
     float d[11];             // minimum per cell position (3 columns each, the last one 2)
     float k[3];              // minimum per column position inside its cell
 };
 
-// One 32-column block of scores: folds its eleven 3-column cell minima into w.d and the minima of
-// the three in-cell column positions into w.k; returns the block minimum.  A column that could be
-// the argmin is thereby pinned to (listed block) x (cell position) x (position in the cell).
-__device__ __forceinline__ float fold_block(Sweep &w, const uint32_t (&u)[32])
+// One 32-column block of scores (block `b` of its chunk): folds its eleven 3-column cell minima into
+// w.d, the minima of the three in-cell column positions into w.k and the block minimum into w.bb[b];
+// returns the block minimum.  A column that could be the argmin is thereby pinned to
+// (listed chunk) x (block of the chunk) x (cell position) x (position in the cell).
+__device__ __forceinline__ float fold_block(Sweep &w, const uint32_t (&u)[32], int b)
 {
     float t[11];
 #pragma unroll
@@ -200,10 +203,12 @@ __device__ __forceinline__ float fold_block(Sweep &w, const uint32_t (&u)[32])
         if (c < 2) m = fminf(m, __uint_as_float(u[30 + c]));      // the last cell has two columns
         w.k[c] = m;
     }
-    return min3(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])), t[9], t[10]);
+    const float m = min3(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])), t[9], t[10]);
+    w.bb[b] = fminf(w.bb[b], m);
+    return m;
 }
 
-// Keep a block's minimum if it is within the window of the running minimum.
+// Keep a chunk's minimum if it is within the window of the running minimum.
 // Branch-free: the value is always written to the next free slot and the slot
 // is claimed only when it belongs on the list; slot kListCap is scratch once
 // the list has overflowed.
@@ -524,6 +529,7 @@ encode_tensor_kernel(const Params p)
 #pragma unroll
                 for (int q = 0; q < 11; ++q) w.d[q] = INFINITY;
                 w.k[0] = w.k[1] = w.k[2] = INFINITY;
+                w.bb[0] = w.bb[1] = w.bb[2] = w.bb[3] = INFINITY;
                 const bool force_scan = !(zmax < 60000.0f) || !(w.win < INFINITY);
 
 #pragma unroll 1
@@ -531,7 +537,7 @@ encode_tensor_kernel(const Params p)
                     if (c == S - 1 && w.cnt > 0) {
                         // Before the last chunk the running winner is the final one most of the time:
                         // start fetching its codeword while the MMA chain runs.
-                        int pb = 0, pq = 0, pk = 0;
+                        int pb = 0, pq = 0, pk = 0, pbb = 0;
 #pragma unroll
                         for (int e = kListCap - 1; e >= 0; --e)
                             if (e < w.cnt && list_v[e * kRowsPerPass] == w.m1) pb = list_i[e * kRowsPerPass];
@@ -540,7 +546,10 @@ encode_tensor_kernel(const Params p)
                             if (w.d[q] == w.m1) pq = q;
                         if (w.k[1] == w.m1) pk = 1;
                         if (w.k[2] == w.m1) pk = 2;
-                        const int pj = min(pb * 32 + 3 * pq + pk, s.K - 1);
+#pragma unroll
+                        for (int i = 3; i > 0; --i)
+                            if (w.bb[i] == w.m1) pbb = i;
+                        const int pj = min(pb * 128 + pbb * 32 + 3 * pq + pk, s.K - 1);
                         asm volatile("prefetch.global.L1 [%0];" ::"l"(cbr + (size_t)pj * 32));
                     }
                     ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag);
@@ -548,26 +557,22 @@ encode_tensor_kernel(const Params p)
                     ++chunk_use;
                     if (!ok) break;
                     tc_fence_after();
-                    // Four 32-column blocks, three of them in flight at once; the fourth is asked for as
-                    // soon as the first has been reduced, and the accumulator goes back to the MMA issuer
-                    // when it has landed.
-                    uint32_t ua[32], ub[32], uc[32];
+                    // All four 32-column blocks are asked for at once and the accumulator goes back to
+                    // the MMA issuer as soon as they have landed: the reduction below runs while the
+                    // next chain computes.
+                    uint32_t ua[32], ub[32], uc[32], ud[32];
                     tmem_ld32_issue(taddr, ua);
                     tmem_ld32_issue(taddr + 32, ub);
                     tmem_ld32_issue(taddr + 64, uc);
-                    tmem_ld_wait3(ua, ub, uc);
-                    const float c0 = fold_block(w, ua);
-                    tmem_ld32_issue(taddr + 96, ua);
-                    const float c1 = fold_block(w, ub);
-                    const float c2 = fold_block(w, uc);
-                    tmem_ld_wait(ua);
+                    tmem_ld32_issue(taddr + 96, ud);
+                    tmem_ld_wait4(ua, ub, uc, ud);
                     tc_fence_before();
                     mbar_arrive(BAR(kBarAccFree + tile));        // the accumulator may be overwritten
-                    const float c3 = fold_block(w, ua);
-                    list_block(w, c0, c * 4, list_v, list_i, kRowsPerPass);
-                    list_block(w, c1, c * 4 + 1, list_v, list_i, kRowsPerPass);
-                    list_block(w, c2, c * 4 + 2, list_v, list_i, kRowsPerPass);
-                    list_block(w, c3, c * 4 + 3, list_v, list_i, kRowsPerPass);
+                    const float c0 = fold_block(w, ua, 0);
+                    const float c1 = fold_block(w, ub, 1);
+                    const float c2 = fold_block(w, uc, 2);
+                    const float c3 = fold_block(w, ud, 3);
+                    list_block(w, fminf(min3(c0, c1, c2), c3), c, list_v, list_i, kRowsPerPass);
                 }
                 if (!ok) break;
                 // take the residual back
@@ -593,8 +598,13 @@ encode_tensor_kernel(const Params p)
                         if (live && !found && fv == m1) { found = true; b1 = fi; }
                     }
                 }
-                uint32_t qmask = 0u, kmask = 0u;
-                int q1 = 0, k1 = 0;
+                uint32_t qmask = 0u, kmask = 0u, bmask = 0u;
+                int q1 = 0, k1 = 0, bb1 = 0;
+#pragma unroll
+                for (int i = 3; i >= 0; --i) {
+                    if (w.bb[i] <= lim) bmask |= 1u << i;
+                    if (w.bb[i] == m1) bb1 = i;
+                }
 #pragma unroll
                 for (int q = 10; q >= 0; --q) {
                     if (w.d[q] <= lim) qmask |= 1u << q;
@@ -605,10 +615,11 @@ encode_tensor_kernel(const Params p)
                     if (w.k[c] <= lim) kmask |= 1u << c;
                     if (w.k[c] == m1) k1 = c;
                 }
-                const int j1 = b1 * 32 + 3 * q1 + k1;
+                const int j1 = b1 * 128 + bb1 * 32 + 3 * q1 + k1;
                 // (a padded column scores 60000: if nothing real scored less, scan everything)
                 const bool scan_all = force_scan || cnt == 0 || cnt > kListCap || !(m1 < 59000.0f);
-                const bool unique = nlisted == 1 && (qmask & (qmask - 1u)) == 0u && (kmask & (kmask - 1u)) == 0u && j1 < s.K;
+                const bool unique = nlisted == 1 && (qmask & (qmask - 1u)) == 0u && (kmask & (kmask - 1u)) == 0u &&
+                                    (bmask & (bmask - 1u)) == 0u && j1 < s.K;
                 const bool flagged = !deg && (scan_all || !unique);
                 int bj = j1 < s.K ? j1 : 0;
                 // Rows with more than one candidate: the whole warp re-scores the candidate columns of
@@ -626,6 +637,7 @@ encode_tensor_kernel(const Params p)
                     const int cnt_s = __shfl_sync(0xFFFFFFFFu, cnt, src);
                     const uint32_t qmask_s = __shfl_sync(0xFFFFFFFFu, qmask, src);
                     const uint32_t kmask_s = __shfl_sync(0xFFFFFFFFu, kmask, src);
+                    const uint32_t bmask_s = __shfl_sync(0xFFFFFFFFu, bmask, src);
                     const bool all_s = __shfl_sync(0xFFFFFFFFu, (int)scan_all, src) != 0;
                     const int row_s = rloc - lane + src;
                     const int lq = lane >= 30 ? 10 : lane / 3;
@@ -641,10 +653,13 @@ encode_tensor_kernel(const Params p)
                         for (int e = 0; e < cnt_s; ++e) {
                             const float fv = reinterpret_cast<const float *>(smem + kOffListV)[e * kRowsPerPass + row_s];
                             if (!(fv <= lim_s)) continue;                              // warp-uniform
-                            const int j = (int)reinterpret_cast<const uint16_t *>(smem + kOffListI)[e * kRowsPerPass + row_s] * 32 + lane;
-                            if (mine && j < s.K) {
-                                const float dj = exact_distance(zs, cbr + (size_t)j * 32);
-                                if (dj < bv) { bv = dj; bi = j; }
+                            const int j0 = (int)reinterpret_cast<const uint16_t *>(smem + kOffListI)[e * kRowsPerPass + row_s] * 128 + lane;
+                            for (int i = 0; i < 4; ++i) {
+                                const int j = j0 + 32 * i;
+                                if (((bmask_s >> i) & 1u) && mine && j < s.K) {     // (the block test is warp-uniform)
+                                    const float dj = exact_distance(zs, cbr + (size_t)j * 32);
+                                    if (dj < bv) { bv = dj; bi = j; }
+                                }
                             }
                         }
                     }

@@ -89,7 +89,9 @@ const char *rvq_status_string(int code);
 int rvq_version(void);
 
 /* Diagnostic: number of kernels this library has launched in this process so
- * far (the only process-wide state it keeps). */
+ * far.  (Process-wide state of the library: this counter, and the per-device
+ * address of the built-in scratch array that rvq_ema_update_static resolves on
+ * its first call.) */
 uint64_t rvq_launch_count(void);
 
 /* Bytes of one head vector's codes in the configured storage form
@@ -124,6 +126,12 @@ size_t rvq_workspace_bytes(const rvq_config *cfg /* host */, int64_t n);
  *   prepared     in   block written by rvq_prepare_codebooks for these codebooks
  *   codes        out  see "codes" above; rvq_code_bytes() * n bytes
  *   std_f16      out  binary16 rounding of s (the scaling itself uses s unrounded)
+ *   stage_energy out  optional (may be NULL): float32 [R], overwritten; entry r is the sum over
+ *                     all groups of all n head vectors of ||z_{r+1}||^2, the squared norm of the
+ *                     residual that stage r leaves, in scaled units (after the division by s).
+ *                     Entry R-1 is the quantization error of the batch: the quantity Section 3
+ *                     watches while the codebooks are learnt.  Float32 atomics: the order of
+ *                     the additions, and so the last bits, vary from call to call.
  *   workspace         rvq_workspace_bytes(cfg, n) bytes, 256-byte aligned; may be
  *                     NULL when that size is 0
  *   status            optional counters (may be NULL)
@@ -131,7 +139,7 @@ size_t rvq_workspace_bytes(const rvq_config *cfg /* host */, int64_t n);
  */
 int rvq_encode(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
                const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-               void *workspace, size_t workspace_bytes, rvq_status *status,
+               float *stage_energy, void *workspace, size_t workspace_bytes, rvq_status *status,
                void *stream /* cudaStream_t */);
 
 /*
@@ -140,6 +148,7 @@ int rvq_encode(const rvq_config *cfg /* host */, const void *x, int64_t n, int64
  * batch).  Results are those of rvq_encode followed by rvq_ema_stats on the
  * codes it produced: the residual entering every stage is already in registers
  * when its code is chosen, so x is not read and re-scaled a second time.
+ *   stage_energy out  optional [R], as under rvq_encode
  *   batch_count  out  float32 [R][K]             (overwritten)
  *   batch_sum    out  float32 [R][K][group_dim]  (overwritten; 16-byte aligned)
  *   workspace         rvq_workspace_bytes(cfg, n) bytes, 256-byte aligned
@@ -147,8 +156,8 @@ int rvq_encode(const rvq_config *cfg /* host */, const void *x, int64_t n, int64
  */
 int rvq_encode_stats(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
                      const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-                     float *batch_count, float *batch_sum, void *workspace, size_t workspace_bytes,
-                     rvq_status *status, void *stream /* cudaStream_t */);
+                     float *stage_energy, float *batch_count, float *batch_sum, void *workspace,
+                     size_t workspace_bytes, rvq_status *status, void *stream /* cudaStream_t */);
 
 /*
  * The same encode computed entirely in float32 on the CUDA cores (every
@@ -159,7 +168,7 @@ int rvq_encode_stats(const rvq_config *cfg /* host */, const void *x, int64_t n,
  */
 int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
                      const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-                     rvq_status *status, void *stream /* cudaStream_t */);
+                     float *stage_energy, rvq_status *status, void *stream /* cudaStream_t */);
 
 /*
  * Decode (Section 2.2, last sentence; Section 3.2).  For every head vector and
@@ -216,8 +225,8 @@ int rvq_rope_table(int32_t dim, double base, int32_t positions, float *cos_sin /
                    void *stream /* cudaStream_t */);
 
 /*
- * One EMA codebook update (Section 3: "update them using exponential moving
- * average with a decay factor of 0.99"; Section 2.1: EMA in place of the
+ * One EMA codebook update (Section 3: the codebooks follow an exponential moving
+ * average with decay 0.99; Section 2.1: EMA in place of the
  * codebook loss).  With n_r[j] the number of group rows whose stage-r code is j
  * and m_r[j] the sum of their stage-r inputs z_r (scaled space, rebuilt from x,
  * the codes and the codebooks passed in):
@@ -270,17 +279,18 @@ int rvq_ema_apply(const rvq_config *cfg /* host */, const float *batch_count,
  *   codebooks, prepared   in/out
  *   ema_count, ema_sum    in/out  N [R][K] and M [R][K][group_dim]
  *   codes, std_f16        out     the batch encoded with the codebooks as they came in
+ *   stage_energy          out     optional [R], as under rvq_encode: the loss curve of the learning loop
  *   workspace                     rvq_workspace_bytes(cfg, n) bytes, 256-byte aligned
  */
 int rvq_learn_step(const rvq_config *cfg /* host */, const void *x, int64_t n, int64_t x_row_stride,
                    float *codebooks, void *prepared, float *ema_count, float *ema_sum, void *codes,
-                   uint16_t *std_f16, float decay, float eps, void *workspace, size_t workspace_bytes,
-                   rvq_status *status, void *stream /* cudaStream_t */);
+                   uint16_t *std_f16, float *stage_energy, float decay, float eps, void *workspace,
+                   size_t workspace_bytes, rvq_status *status, void *stream /* cudaStream_t */);
 
 /*
- * k-means initialisation of the codebooks on one batch (Section 3: "we
- * initialize each codebook using k-means"; the paper gives no further detail,
- * so the variant is this library's: plain Lloyd iterations).  Stage r works on
+ * k-means initialisation of the codebooks on one batch (Section 3: every codebook
+ * starts from a k-means run; the paper gives no further detail, so the
+ * variant is this library's: plain Lloyd iterations).  Stage r works on
  * the stage-r inputs of the batch -- the scaled group rows minus the centroids
  * chosen at the earlier stages -- starting from the rows seed_rows[r][0..K) of
  * that input: `iterations` times every row is assigned to its nearest centroid

@@ -105,7 +105,7 @@ double rvq_oracle_f16_bits_to_f64(uint16_t h)
     return s ? -v : v;
 }
 
-/* Section 2.2 "scale x by its standard deviation": mu = mean(x),
+/* Section 2.2 (x is scaled by its own standard deviation): mu = mean(x),
  * s = sqrt(sum((x-mu)^2) / (d - ddof)).  x itself is not centred. */
 static double vector_std(const double *x, int d, int ddof)
 {

@@ -55,11 +55,11 @@ def _load() -> ctypes.CDLL:
     lib.rvq_prepare_codebooks.restype = ctypes.c_int
     lib.rvq_prepare_codebooks.argtypes = [cfgp, vp, vp, vp]
     lib.rvq_encode.restype = ctypes.c_int
-    lib.rvq_encode.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.rvq_encode.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.rvq_encode_exact.restype = ctypes.c_int
-    lib.rvq_encode_exact.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp]
+    lib.rvq_encode_exact.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp]
     lib.rvq_encode_stats.restype = ctypes.c_int
-    lib.rvq_encode_stats.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.rvq_encode_stats.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.rvq_decode.restype = ctypes.c_int
     lib.rvq_decode.argtypes = [cfgp, vp, vp, i64, vp, vp, vp, i64, vp, vp]
     lib.rvq_ema_update.restype = ctypes.c_int
@@ -80,7 +80,7 @@ def _load() -> ctypes.CDLL:
     lib.rvq_decode_rope.argtypes = [cfgp, vp, vp, i64, vp, vp, vp, ctypes.c_int32, vp, ctypes.c_int32,
                                     ctypes.c_int32, vp, i64, vp, vp]
     lib.rvq_learn_step.restype = ctypes.c_int
-    lib.rvq_learn_step.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
+    lib.rvq_learn_step.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
                                    vp, sz, vp, vp]
     lib.rvq_kmeans_workspace_bytes.restype = sz
     lib.rvq_kmeans_workspace_bytes.argtypes = [cfgp, i64]
@@ -148,29 +148,29 @@ def rvq_prepare_codebooks(cfg, codebooks, prepared, stream=None, check=True) -> 
 
 
 def rvq_encode(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, workspace=None,
-               workspace_bytes=0, status=None, stream=None, check=True) -> int:
+               workspace_bytes=0, status=None, stream=None, check=True, stage_energy=None) -> int:
     rc = lib.rvq_encode(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
-                        _ptr(codes), _ptr(std_f16), _ptr(workspace), workspace_bytes, _ptr(status),
-                        _stream(stream))
+                        _ptr(codes), _ptr(std_f16), _ptr(stage_energy), _ptr(workspace), workspace_bytes,
+                        _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_encode")
     return rc
 
 
 def rvq_encode_stats(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, batch_count, batch_sum,
-                     workspace, workspace_bytes, status=None, stream=None, check=True) -> int:
+                     workspace, workspace_bytes, status=None, stream=None, check=True, stage_energy=None) -> int:
     rc = lib.rvq_encode_stats(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
-                              _ptr(codes), _ptr(std_f16), _ptr(batch_count), _ptr(batch_sum), _ptr(workspace),
-                              workspace_bytes, _ptr(status), _stream(stream))
+                              _ptr(codes), _ptr(std_f16), _ptr(stage_energy), _ptr(batch_count), _ptr(batch_sum),
+                              _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_encode_stats")
     return rc
 
 
 def rvq_encode_exact(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status=None,
-                     stream=None, check=True) -> int:
+                     stream=None, check=True, stage_energy=None) -> int:
     rc = lib.rvq_encode_exact(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
-                              _ptr(codes), _ptr(std_f16), _ptr(status), _stream(stream))
+                              _ptr(codes), _ptr(std_f16), _ptr(stage_energy), _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_encode_exact")
     return rc
@@ -251,10 +251,11 @@ def rvq_decode_rope(cfg, codes, std_f16, n, codebooks, prepared, position, vecto
 
 
 def rvq_learn_step(cfg, x, n, x_row_stride, codebooks, prepared, ema_count, ema_sum, codes, std_f16,
-                   decay, eps, workspace, workspace_bytes, status=None, stream=None, check=True) -> int:
+                   decay, eps, workspace, workspace_bytes, status=None, stream=None, check=True,
+                   stage_energy=None) -> int:
     """Encode the batch, update N, M and the codebooks from its assignments, rebuild the prepared block."""
     rc = lib.rvq_learn_step(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
-                            _ptr(ema_count), _ptr(ema_sum), _ptr(codes), _ptr(std_f16), decay, eps,
+                            _ptr(ema_count), _ptr(ema_sum), _ptr(codes), _ptr(std_f16), _ptr(stage_energy), decay, eps,
                             _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_learn_step")

@@ -1,5 +1,7 @@
 // extern "C" boundary of the RVQ library: argument checks on the host, then
-// dispatch to the kernels.  No allocation, no synchronisation, no global state.
+// dispatch to the kernels.  No allocation, no synchronisation.  Process-wide
+// state: the launch counter below, and (in ema.cu) the per-device address of
+// the built-in scratch array of rvq_ema_update_static.
 #include "prepared.cuh"
 
 #include <atomic>
@@ -103,7 +105,8 @@ size_t rvq_workspace_bytes(const rvq_config *cfg, int64_t n)
 
 static int encode_common(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
                          const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-                         rvq_status *status, void *stream, bool allow_tensor)
+                         float *stage_energy, rvq_status *status, void *stream, bool allow_tensor,
+                         uint32_t *stat_cnt = nullptr, float *stat_sum = nullptr)
 {
     Shape s;
     int rc = make_shape(cfg, &s);
@@ -111,24 +114,27 @@ static int encode_common(const rvq_config *cfg, const void *x, int64_t n, int64_
     if ((rc = check_rows(s, x, n, x_row_stride)) != RVQ_OK) return rc;
     if (!codebooks || !prepared || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
     if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    if (stage_energy && cudaMemsetAsync(stage_energy, 0, (size_t)s.R * sizeof(float), (cudaStream_t)stream) != cudaSuccess)
+        return RVQ_ERR_LAUNCH;
     if (allow_tensor && encode_tensor_supported(s))
         return launch_encode_tensor(s, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status,
-                                    (cudaStream_t)stream);
-    return launch_encode_scalar(s, x, n, x_row_stride, codebooks, codes, std_f16, status, (cudaStream_t)stream);
+                                    (cudaStream_t)stream, stat_cnt, stat_sum, stage_energy);
+    return launch_encode_scalar(s, x, n, x_row_stride, codebooks, codes, std_f16, status, (cudaStream_t)stream,
+                                stage_energy);
 }
 
 int rvq_encode(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
                const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-               void *workspace, size_t workspace_bytes, rvq_status *status, void *stream)
+               float *stage_energy, void *workspace, size_t workspace_bytes, rvq_status *status, void *stream)
 {
     (void)workspace; (void)workspace_bytes;
-    return encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, stream, true);
+    return encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, stage_energy, status, stream, true);
 }
 
 int rvq_encode_stats(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
                      const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-                     float *batch_count, float *batch_sum, void *workspace, size_t workspace_bytes,
-                     rvq_status *status, void *stream)
+                     float *stage_energy, float *batch_count, float *batch_sum, void *workspace,
+                     size_t workspace_bytes, rvq_status *status, void *stream)
 {
     Shape s;
     int rc = make_shape(cfg, &s);
@@ -138,7 +144,7 @@ int rvq_encode_stats(const rvq_config *cfg, const void *x, int64_t n, int64_t x_
     if (workspace_bytes < ema_stats_scratch_bytes(s)) return RVQ_ERR_WORKSPACE;
     if (!encode_tensor_supported(s)) {
         // shapes without the fused kernel: encode, then the separate statistics pass
-        rc = encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, stream, true);
+        rc = encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, stage_energy, status, stream, true);
         if (rc != RVQ_OK) return rc;
         return launch_ema_stats(s, x, n, x_row_stride, codes, codebooks, batch_count, batch_sum, workspace,
                                 status, (cudaStream_t)stream);
@@ -152,16 +158,17 @@ int rvq_encode_stats(const rvq_config *cfg, const void *x, int64_t n, int64_t x_
     if (cudaMemsetAsync(cnt, 0, (size_t)bins * sizeof(uint32_t), st) != cudaSuccess ||
         cudaMemsetAsync(batch_sum, 0, (size_t)bins * s.gd * sizeof(float), st) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
-    rc = launch_encode_tensor(s, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, st, cnt, batch_sum);
+    rc = encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, stage_energy, status, stream, true,
+                       cnt, batch_sum);
     if (rc != RVQ_OK) return rc;
     return launch_counts_to_float(cnt, batch_count, bins, st);
 }
 
 int rvq_encode_exact(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
                      const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
-                     rvq_status *status, void *stream)
+                     float *stage_energy, rvq_status *status, void *stream)
 {
-    return encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status, stream, false);
+    return encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, stage_energy, status, stream, false);
 }
 
 int rvq_decode(const rvq_config *cfg, const void *codes, const uint16_t *std_f16, int64_t n,
@@ -272,8 +279,8 @@ int rvq_ema_update(const rvq_config *cfg, const void *x, int64_t n, int64_t x_ro
 
 int rvq_learn_step(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
                    float *codebooks, void *prepared, float *ema_count, float *ema_sum, void *codes,
-                   uint16_t *std_f16, float decay, float eps, void *workspace, size_t workspace_bytes,
-                   rvq_status *status, void *stream)
+                   uint16_t *std_f16, float *stage_energy, float decay, float eps, void *workspace,
+                   size_t workspace_bytes, rvq_status *status, void *stream)
 {
     Shape s;
     int rc = make_shape(cfg, &s);
@@ -287,8 +294,8 @@ int rvq_learn_step(const rvq_config *cfg, const void *x, int64_t n, int64_t x_ro
     float *bc = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s));
     float *bs = reinterpret_cast<float *>(ws + ema_stats_scratch_bytes(s) +
                                           ((size_t)s.R * s.K * sizeof(float) + 255) / 256 * 256);
-    rc = rvq_encode_stats(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, bc, bs, workspace,
-                          workspace_bytes, status, stream);
+    rc = rvq_encode_stats(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, stage_energy, bc, bs,
+                          workspace, workspace_bytes, status, stream);
     if (rc != RVQ_OK) return rc;
     rc = launch_ema_apply(s, bc, bs, codebooks, ema_count, ema_sum, decay, eps, (cudaStream_t)stream);
     if (rc != RVQ_OK) return rc;

@@ -12,8 +12,10 @@ template <int GD>
 __global__ void __launch_bounds__(128)
 encode_scalar_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t stride,
                      const float *__restrict__ cb, void *__restrict__ codes,
-                     uint16_t *__restrict__ std16, rvq_status *st, int vpb)
+                     uint16_t *__restrict__ std16, rvq_status *st, int vpb, float *energy)
 {
+    __shared__ float e_stage[16];                       // per-stage residual energy of this block's rows
+    if (threadIdx.x < 16) e_stage[threadIdx.x] = 0.0f;
     extern __shared__ __align__(16) float smem[];
     float *xs = smem;                                   // [vpb][dim]
     float *cbs = xs + vpb * s.dim;                      // [kChunk][GD]
@@ -68,8 +70,15 @@ encode_scalar_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t str
             float4 ev = __ldg(e + q);
             z[4 * q] -= ev.x; z[4 * q + 1] -= ev.y; z[4 * q + 2] -= ev.z; z[4 * q + 3] -= ev.w;
         }
+        if (energy && gv < n) {
+            float e2 = 0.0f;
+#pragma unroll
+            for (int i = 0; i < GD; ++i) e2 = fmaf(z[i], z[i], e2);
+            atomicAdd(&e_stage[r], e2);
+        }
     }
     __syncthreads();
+    if (energy && tid < s.R) atomicAdd(energy + tid, e_stage[tid]);
 
     // emit codes (Section 3.2 storage) and the half-precision deviation
     if (s.bits == 16) {
@@ -105,7 +114,7 @@ encode_scalar_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t str
 
 template <int GD>
 static int launch_gd(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
-                     void *codes, uint16_t *std16, rvq_status *st, cudaStream_t stream)
+                     void *codes, uint16_t *std16, rvq_status *st, cudaStream_t stream, float *energy)
 {
     const int vpb = 128 / s.G > 0 ? 128 / s.G : 1;
     const int threads = vpb * s.G;
@@ -115,19 +124,19 @@ static int launch_gd(const Shape &s, const void *x, int64_t n, int64_t stride, c
     if (blocks > 0x7FFFFFFF) return RVQ_ERR_UNSUPPORTED;
     if (smem > 48 * 1024)
         cudaFuncSetAttribute(encode_scalar_kernel<GD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    encode_scalar_kernel<GD><<<(unsigned)blocks, threads, smem, stream>>>(s, x, n, stride, cb, codes, std16, st, vpb);
+    encode_scalar_kernel<GD><<<(unsigned)blocks, threads, smem, stream>>>(s, x, n, stride, cb, codes, std16, st, vpb, energy);
     return check_launch();
 }
 
 int launch_encode_scalar(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
-                         void *codes, uint16_t *std16, rvq_status *st, cudaStream_t stream)
+                         void *codes, uint16_t *std16, rvq_status *st, cudaStream_t stream, float *energy)
 {
     if (n == 0) return RVQ_OK;
     switch (s.gd) {
-    case 8: return launch_gd<8>(s, x, n, stride, cb, codes, std16, st, stream);
-    case 16: return launch_gd<16>(s, x, n, stride, cb, codes, std16, st, stream);
-    case 32: return launch_gd<32>(s, x, n, stride, cb, codes, std16, st, stream);
-    case 64: return launch_gd<64>(s, x, n, stride, cb, codes, std16, st, stream);
+    case 8: return launch_gd<8>(s, x, n, stride, cb, codes, std16, st, stream, energy);
+    case 16: return launch_gd<16>(s, x, n, stride, cb, codes, std16, st, stream, energy);
+    case 32: return launch_gd<32>(s, x, n, stride, cb, codes, std16, st, stream, energy);
+    case 64: return launch_gd<64>(s, x, n, stride, cb, codes, std16, st, stream, energy);
     default: return RVQ_ERR_UNSUPPORTED;
     }
 }

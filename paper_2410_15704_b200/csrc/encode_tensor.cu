@@ -73,12 +73,18 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait; returns false (and raises the CTA's abort flag) when it gives up.
+// Bounded wait; returns false (and raises the CTA's abort flag) when it gives up.  A phase that has
+// completed already is recognised by the non-blocking test (a plain shared-memory read); only a
+// phase still pending goes through the suspending form.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
 {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
 #pragma unroll 1
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
-        uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
@@ -278,6 +284,7 @@ struct Params {
     int tiles;          // 128-row tiles in the whole problem
     uint32_t *stat_cnt; // optional EMA statistics of this batch: counts [R][K] ...
     float *stat_sum;    // ... and sums of the stage inputs [R][K][32]; both null when not wanted
+    float *energy;      // optional [R]: sum over the rows of the squared norm of what each stage leaves
 };
 
 // The tiles of one CTA: a contiguous run, done in `rounds` rounds of nearly equal size (<= kTiles).
@@ -442,14 +449,26 @@ encode_tensor_kernel(const Params p)
                 const int eb = s.elem_bytes, ppv = s.dim * eb / 16;          // pieces per vector (>= 4)
                 const int64_t v_first = (row0 + q4 * 32) / G;
                 float *scr = reinterpret_cast<float *>(smem + kOffZ) + (rloc - lane);
-                for (int c = lane; c < (32 / G) * ppv; c += 32) {
-                    const int vl = c / ppv, off = c - vl * ppv;
-                    const int64_t vv = v_first + vl;
-                    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-                    if (vv < p.n)
-                        val = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(p.x) + vv * p.stride * eb) + off);
-                    const int k = (vl * ppv + (off ^ (vl & 7 & (ppv - 1)))) * 4;
-                    *reinterpret_cast<uint4 *>(scr + (k >> 5) * kRowsPerPass + (k & 31)) = val;
+                // (four loads in flight per lane: a 16-bit head vector of 128 channels is 16 pieces, so the
+                // 8 vectors of a warp are 4 pieces per lane)
+                const int npieces = (32 / G) * ppv;
+                for (int c0 = 0; c0 < npieces; c0 += 128) {
+                    uint4 val[4];
+                    int kk[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = c0 + 32 * u + lane;
+                        const int vl = c / ppv, off = c - vl * ppv;
+                        const int64_t vv = v_first + vl;
+                        val[u] = make_uint4(0u, 0u, 0u, 0u);
+                        if (c < npieces && vv < p.n)
+                            val[u] = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(p.x) + vv * p.stride * eb) + off);
+                        kk[u] = (vl * ppv + (off ^ (vl & 7 & (ppv - 1)))) * 4;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (c0 + 32 * u + lane < npieces)
+                            *reinterpret_cast<uint4 *>(scr + (kk[u] >> 5) * kRowsPerPass + (kk[u] & 31)) = val[u];
                 }
                 __syncwarp();
                 const int vl = lane / G, sw = vl & 7 & (ppv - 1);
@@ -696,6 +715,17 @@ encode_tensor_kernel(const Params p)
                         for (int k = 0; k < 8; ++k) z[8 * q + k] -= ev[k];
                     }
                 }
+                if (p.energy) {
+                    // squared norm of the residual leaving this stage (scaled units), summed over the
+                    // warp's rows: one atomic per warp and stage
+                    float e2 = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) e2 = fmaf(z[i], z[i], e2);
+                    if (!valid) e2 = 0.0f;
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) e2 += __shfl_xor_sync(0xFFFFFFFFu, e2, off);
+                    if (lane == 0) atomicAdd(p.energy + r, e2);
+                }
                 codes_s[rloc * 16 + r] = (uint16_t)bj;
             }
             if (!ok) break;
@@ -758,7 +788,7 @@ bool encode_tensor_supported(const Shape &s)
 
 int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
                          const void *prepared, void *codes, uint16_t *std16, rvq_status *st,
-                         cudaStream_t stream, uint32_t *stat_cnt, float *stat_sum)
+                         cudaStream_t stream, uint32_t *stat_cnt, float *stat_sum, float *energy)
 {
     if (n == 0) return RVQ_OK;
     const int64_t rows = n * s.G;
@@ -770,7 +800,8 @@ int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t strid
         return RVQ_ERR_DEVICE;
     if (cudaFuncSetAttribute(encode_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
-    Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)tiles, stat_cnt, stat_sum};
+    Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)tiles, stat_cnt, stat_sum,
+             energy};
     const int64_t groups = (tiles + kTiles - 1) / kTiles;
     const int grid = (int)(groups < sms ? groups : sms);
     encode_tensor_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);

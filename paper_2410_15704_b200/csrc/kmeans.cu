@@ -1,5 +1,5 @@
-// k-means initialisation of the codebooks (Section 3: "we initialize each
-// codebook using k-means"), stage after stage on that stage's inputs.
+// k-means initialisation of the codebooks (Section 3: every codebook starts
+// from a k-means run on the first batch), stage after stage on that stage's inputs.
 //
 // The scaled group rows of the batch are written once to a float32 buffer
 // [n][G][32]; stage r then runs Lloyd's iterations on it: the assignment is the

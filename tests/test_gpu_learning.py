@@ -121,3 +121,61 @@ def test_kmeans_init_on_key_like_data():
     torch.cuda.synchronize()
     assert_codes_match(w.x, codes_to_numpy(cfg, b.codes, w.n), got.astype(np.float32), w.layout)
     print(f"k-means (key-like): residual energy seeds {e0:.4f}, 5 iterations {e_got:.4f}, oracle {e_ref:.4f}")
+
+
+def gpu_assign(cfg_r, x, n, cbs):
+    """Codes the GPU encoder gives `x` with the codebooks `cbs` (float32 [r][K][32])."""
+    b = rvq.alloc_buffers(cfg_r, n, cbs)
+    rvq.rvq_encode(cfg_r, x_to_device(x, cfg_r.x_dtype), n, cfg_r.dim, b.codebooks, b.prepared, b.codes, b.std,
+                   b.workspace, b.workspace_bytes, b.status)
+    torch.cuda.synchronize()
+    return codes_to_numpy(cfg_r, b.codes, n)
+
+
+@pytest.mark.parametrize("layout", [rvq_synth.CONTIGUOUS, rvq_synth.STRIDED])
+def test_kmeans_lloyd_iterations_teacher_forced(layout):
+    """Single Lloyd iterations checked centroid by centroid.  An iteration is an assignment followed
+    by cluster means; the assignment the GPU makes from given centroids is the encoder's (checked
+    against the oracle's argmin), and with that assignment fixed the means have one right answer,
+    which the oracle computes: every centroid must agree within 1e-3.  Done for the first and the
+    second iteration of stage 0 and for the first iteration of stage 1 (whose rows are what stage 0
+    leaves) on key-like data, where free-running runs may part at near ties."""
+    w = rvq_synth.key_cache(tokens=512, depth=2, size=64)
+    w.layout = layout
+    K, G = 64, w.groups
+    g = np.random.default_rng(91)
+    seeds = np.stack([g.choice(w.n * G, K, replace=False) for _ in range(2)]).astype(np.int64)
+
+    def cfg_for(depth):
+        return rvq.make_config(w.dim, 32, layout, depth, K, 16, rvq.BF16, 0)
+
+    z0 = oracle.scaled_groups(w.x, 32, layout).reshape(-1, 32)           # stage-0 rows [n*G][32], float64
+
+    def means(rows, codes, before):
+        out = before.astype(np.float64).copy()
+        for j in range(K):
+            sel = codes == j
+            if sel.any():
+                out[j] = rows[sel].mean(axis=0)
+        return out
+
+    prev, _, _ = gpu_kmeans(cfg_for(1), w.x, w.n, seeds[:1], 0)          # the seed centroids as the GPU holds them
+    for it in (1, 2):
+        got, _, _ = gpu_kmeans(cfg_for(1), w.x, w.n, seeds[:1], it)
+        codes = gpu_assign(cfg_for(1), w.x, w.n, prev.astype(np.float32))
+        assert_codes_match(w.x, codes, prev.astype(np.float32), layout)
+        want = means(z0, codes.reshape(-1), prev[0])
+        assert np.abs(got[0] - want).max() <= RECON_TOL, f"stage 0, iteration {it}"
+        prev = got
+    # stage 1 after one iteration per stage: rows = stage-0 rows minus the centroid stage 0 assigned them
+    got2, _, _ = gpu_kmeans(cfg_for(2), w.x, w.n, seeds, 1)
+    cb0 = got2[0]
+    codes0 = gpu_assign(cfg_for(1), w.x, w.n, cb0[None].astype(np.float32)).reshape(-1)
+    z1 = z0 - cb0[codes0]
+    seed_centroids = z1[seeds[1]]
+    both = np.stack([cb0, seed_centroids]).astype(np.float32)
+    codes = gpu_assign(cfg_for(2), w.x, w.n, both)
+    assert_codes_match(w.x, codes, both, layout)
+    assert np.array_equal(codes[:, :, 0].reshape(-1), codes0)
+    want1 = means(z1, codes[:, :, 1].reshape(-1), seed_centroids)
+    assert np.abs(got2[1] - want1).max() <= RECON_TOL, "stage 1, iteration 1"

@@ -42,26 +42,26 @@ def test_sizes_and_strings():
 def test_bad_configs_are_rejected(kw):
     cfg = rvq.make_config(**kw)
     assert rvq.rvq_code_bytes(cfg) == 0 and rvq.rvq_prepared_bytes(cfg) == 0
-    rc = rvq.lib.rvq_encode(ctypes.byref(cfg), 256, 1, 128, 256, 256, 256, 256, None, 0, None, None)
+    rc = rvq.lib.rvq_encode(ctypes.byref(cfg), 256, 1, 128, 256, 256, 256, 256, None, None, 0, None, None)
     assert rc in (-1, -3)
 
 
 def test_bad_pointers_are_rejected_before_launch():
     cfg = rvq.make_config(code_bits=11)
     c = ctypes.byref(cfg)
-    assert rvq.lib.rvq_encode(c, None, 4, 128, 256, 256, 256, 256, None, 0, None, None) == -1
-    assert rvq.lib.rvq_encode(c, 256, -1, 128, 256, 256, 256, 256, None, 0, None, None) == -1
-    assert rvq.lib.rvq_encode(c, 256, 4, 64, 256, 256, 256, 256, None, 0, None, None) == -1      # stride < dim
-    assert rvq.lib.rvq_encode(c, 260, 4, 128, 256, 256, 256, 256, None, 0, None, None) == -2     # x misaligned
-    assert rvq.lib.rvq_encode(c, 256, 4, 132, 256, 256, 256, 256, None, 0, None, None) == -2     # stride bytes % 16
-    assert rvq.lib.rvq_encode(c, 256, 4, 128, 256, 272, 256, 256, None, 0, None, None) == -2     # prepared % 256
+    assert rvq.lib.rvq_encode(c, None, 4, 128, 256, 256, 256, 256, None, None, 0, None, None) == -1
+    assert rvq.lib.rvq_encode(c, 256, -1, 128, 256, 256, 256, 256, None, None, 0, None, None) == -1
+    assert rvq.lib.rvq_encode(c, 256, 4, 64, 256, 256, 256, 256, None, None, 0, None, None) == -1      # stride < dim
+    assert rvq.lib.rvq_encode(c, 260, 4, 128, 256, 256, 256, 256, None, None, 0, None, None) == -2     # x misaligned
+    assert rvq.lib.rvq_encode(c, 256, 4, 132, 256, 256, 256, 256, None, None, 0, None, None) == -2     # stride bytes % 16
+    assert rvq.lib.rvq_encode(c, 256, 4, 128, 256, 272, 256, 256, None, None, 0, None, None) == -2     # prepared % 256
     assert rvq.lib.rvq_decode(c, 256, 256, 4, 256, 256, None, 128, None, None) == -1
     assert rvq.lib.rvq_decode(c, 256, 256, 4, 256, 256, 264, 128, None, None) == -2
     assert rvq.lib.rvq_ema_update(c, 256, 4, 128, 256, 256, 256, 256, None, 0.99, 1e-5, 256, 16, None, None) == -4
     assert rvq.lib.rvq_ema_update(c, 256, 4, 128, 256, 256, 256, 256, None, 1.5, 1e-5, 256, 1 << 30, None, None) == -1
     # learning step and k-means initialisation
-    assert rvq.lib.rvq_learn_step(c, 256, 4, 128, 256, 256, 256, 256, 256, 256, 0.99, 1e-5, 256, 16, None, None) == -4
-    assert rvq.lib.rvq_learn_step(c, 256, 4, 128, 256, 256, None, 256, 256, 256, 0.99, 1e-5, 256, 1 << 30, None, None) == -1
+    assert rvq.lib.rvq_learn_step(c, 256, 4, 128, 256, 256, 256, 256, 256, 256, None, 0.99, 1e-5, 256, 16, None, None) == -4
+    assert rvq.lib.rvq_learn_step(c, 256, 4, 128, 256, 256, None, 256, 256, 256, None, 0.99, 1e-5, 256, 1 << 30, None, None) == -1
     big = rvq.rvq_kmeans_workspace_bytes(cfg, 1000)
     assert big >= 1000 * 128 * 4 and big % 256 == 0
     assert rvq.lib.rvq_kmeans_init(c, 256, 4, 128, 256, 3, 256, 256, 256, 16, None, None) == -4       # workspace too small

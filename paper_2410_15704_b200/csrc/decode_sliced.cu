@@ -476,6 +476,231 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
     if (bad && st && slice == 0) atomicAdd(&st->bad_codes, bad);   // every slice sees the same codes
 }
 
+// The level-table decoder for the shapes the timings are quoted on: head vectors of four groups of 32
+// (dim 128), depth 8, 16-bit outputs; codes as uint16 or as a packed stream of 10 to 12 bits.  Same
+// tables, same arithmetic and same results as decode_sliced_body<DT, CH, false>; what differs is the
+// instruction count (the loop is issue bound): 32-bit row numbers, table addresses cut out of the
+// code words with one shift and one mask-or each, one scale register per stage for both halves of
+// a table word (dp2a.lo reads bytes 0-1 of it, dp2a.hi bytes 2-3), layout and code width known at
+// compile time, no per-row code range loop unless a code is out of range.
+// SUMMED: the tables whose levels add up within 16 bits per stage parity (prepared.cuh): the table
+// words of the even steps and of the odd steps are added as they are (which parity of stages a
+// thread's even steps are depends on its lane), and scaled once per parity.
+template <int DT, int CH, int LAYOUT, int BITS, bool SUMMED>
+__device__ __forceinline__ void
+decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                   const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
+                   int64_t stride, rvq_status *st, uint8_t *table)
+{
+    constexpr int NS = 32 / CH;                                  // slices
+    if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;
+    constexpr uint32_t kEntry = 2 * CH, kLine = 8 * kEntry;      // bytes per (code, stage) and per code: 128 or 64
+    constexpr int kShift = CH == 8 ? 7 : 6;                      // log2(kLine)
+    const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
+    const uint32_t slice = blockIdx.x % NS, part = blockIdx.x / NS, parts = gridDim.x / NS;
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, rot = lane & 7u;
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256 + (SUMMED ? decode_table_bytes(s.K) : 0)) +
+                           (size_t)slice * s.K * CH;
+        uint4 *dst = reinterpret_cast<uint4 *>(table);
+        for (uint32_t t = tid; t < (uint32_t)s.K * CH; t += kDecThreads) dst[t] = __ldg(src + t);
+    }
+    // this thread visits stage (rot + k) & 7 at step k (the 8 lanes of a quarter warp then touch 8
+    // different bank groups): the scale of that stage in bytes 0 and 3, and the byte offset of its entry
+    uint32_t scale[SUMMED ? 2 : 8], unit[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        if (!SUMMED || k < 2) {
+            const uint32_t sc = SUMMED ? dp->pscale[(rot + k) & 1u] : dp->scale[(rot + k) & 7u];
+            scale[SUMMED ? (k & 1) : k] = sc | (sc << 24);
+        }
+        unit[k] = ((rot + k) & 7u) * kEntry;
+    }
+    const float bias = dp->bias, base = SUMMED ? dp->pbase : dp->base;
+    const float terr = SUMMED ? dp->perr : dp->err;
+    const float exact_above = terr > 0.0f ? 0.9e-3f / terr : INFINITY;
+    const uint32_t Ku = (uint32_t)s.K;
+    __syncthreads();
+
+    const uint32_t rows = (uint32_t)n << 2;                       // the launcher guarantees n * 4 < 2^31
+    const uint32_t smem_table = (uint32_t)__cvta_generic_to_shared(table);
+    uint32_t bad = 0;
+    // The codes and the deviation of a row are fetched one iteration ahead, so that their latency is
+    // spent while the previous row's table entries are gathered.
+    auto fetch = [&](uint32_t row, uint32_t &c0, uint32_t &c1, uint32_t &c2, uint32_t &c3, uint16_t &sdb) {
+        c0 = c1 = c2 = c3 = 0u;
+        sdb = 0;
+        if (row >= rows) return;
+        const uint32_t v = row >> 2, g = row & 3u;
+        sdb = __ldg(std16 + v);
+        if (BITS == 16) {
+            const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + row);
+            c0 = c.x; c1 = c.y; c2 = c.z; c3 = c.w;
+        } else {
+            // the row's 8 codes are 8 * BITS <= 96 consecutive bits of the vector's stream of 32 * BITS
+            // bits, starting at bit g * 8 * BITS: the words that hold them (cut below)
+            constexpr int words = BITS;                                  // 32 * BITS / 32
+            const uint32_t *wv = reinterpret_cast<const uint32_t *>(codes) + (size_t)v * words;
+            const uint32_t wi = (g * (8u * BITS)) >> 5;
+            c0 = __ldg(wv + wi); c1 = __ldg(wv + wi + 1);
+            c2 = wi + 2 < (uint32_t)words ? __ldg(wv + wi + 2) : 0u;
+            c3 = wi + 3 < (uint32_t)words ? __ldg(wv + wi + 3) : 0u;
+        }
+    };
+    uint32_t p0, p1, p2, p3;
+    uint16_t psd;
+    fetch(part * kDecThreads + tid, p0, p1, p2, p3, psd);
+    for (uint32_t row = part * kDecThreads + tid; row - tid < rows; row += parts * kDecThreads) {
+        // (the loop bound keeps whole warps together for the shuffles below)
+        const bool live = row < rows;
+        const uint32_t v = live ? row >> 2 : 0u, g = row & 3u;
+        // the 8 codes of this row as 4 words, stage r in half r
+        uint32_t c0 = p0, c1 = p1, c2 = p2, c3 = p3;
+        const uint16_t sdb = psd;
+        fetch(row + parts * kDecThreads, p0, p1, p2, p3, psd);
+        if (BITS != 16) {
+            // shift the window down to bit 0 and cut the codes out of it at offsets known at compile time
+            const uint32_t sh = (g * (8u * BITS)) & 31u;
+            const uint32_t u0 = __funnelshift_r(c0, c1, sh), u1 = __funnelshift_r(c1, c2, sh);
+            const uint32_t u2 = __funnelshift_r(c2, c3, sh);
+            uint32_t cw[4] = {0u, 0u, 0u, 0u};
+            cut_codes<BITS, true>(u0, u1, u2, 8, cw);
+            c0 = cw[0]; c1 = cw[1]; c2 = cw[2]; c3 = cw[3];
+        }
+        const uint32_t n0 = c0, n1 = c1, n2 = c2, n3 = c3;          // natural order, for the exact route
+        // rotate the 8 halves left by `rot` so that step k finds its code at a fixed place
+        if (rot & 4u) { const uint32_t t0 = c0, t1 = c1; c0 = c2; c1 = c3; c2 = t0; c3 = t1; }
+        if (rot & 2u) { const uint32_t t0 = c0; c0 = c1; c1 = c2; c2 = c3; c3 = t0; }
+        if (rot & 1u) {
+            const uint32_t b0 = __funnelshift_r(c0, c1, 16), b1 = __funnelshift_r(c1, c2, 16);
+            const uint32_t b2 = __funnelshift_r(c2, c3, 16), b3 = __funnelshift_r(c3, c0, 16);
+            c0 = b0; c1 = b1; c2 = b2; c3 = b3;
+        }
+        // codes out of range (never produced by the encoder): counted, read as code 0
+        {
+            const uint32_t m = __vmaxu2(__vmaxu2(c0, c1), __vmaxu2(c2, c3));
+            if (max(m & 0xFFFFu, m >> 16) >= Ku) {
+                uint32_t *cc[4] = {&c0, &c1, &c2, &c3};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t lo = *cc[c] & 0xFFFFu, hi = *cc[c] >> 16;
+                    if (lo >= Ku) { lo = 0; ++bad; }
+                    if (hi >= Ku) { hi = 0; ++bad; }
+                    *cc[c] = lo | (hi << 16);
+                }
+            }
+        }
+        const float sd = __half2float(__ushort_as_half(sdb));      // (0 beyond the last row)
+        // integer sums of level * scale: one 16-bit x 8-bit dot-product instruction per channel and stage,
+        // or (summed levels) plain additions of the table words and two such instructions per channel
+        uint32_t acc[CH], even[CH / 2], odd[CH / 2];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) acc[i] = 0u;
+#pragma unroll
+        for (int i = 0; i < CH / 2; ++i) { even[i] = 0u; odd[i] = 0u; }
+        const uint32_t cwk[4] = {c0, c1, c2, c3};
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            // byte offset of the table line of this step's code: (code << kShift) | unit
+            const uint32_t w = cwk[k >> 1];
+            const uint32_t line = (k & 1) ? ((w >> (16 - kShift)) & (0xFFFFu << kShift)) : ((w << kShift) & (0xFFFFu << kShift));
+            const uint32_t a = smem_table + (line | unit[k]);
+            uint32_t e[CH / 2];
+            if (CH == 8)
+                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(e[0]), "=r"(e[1]), "=r"(e[CH / 2 - 2]), "=r"(e[CH / 2 - 1]) : "r"(a));
+            else
+                asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(e[0]), "=r"(e[1]) : "r"(a));
+#pragma unroll
+            for (int i = 0; i < CH / 2; ++i) {
+                if (SUMMED) {
+                    if (k & 1) odd[i] += e[i]; else even[i] += e[i];
+                } else {
+                    asm("dp2a.lo.u32.u32 %0, %1, %2, %0;" : "+r"(acc[2 * i]) : "r"(e[i]), "r"(scale[k]));
+                    asm("dp2a.hi.u32.u32 %0, %1, %2, %0;" : "+r"(acc[2 * i + 1]) : "r"(e[i]), "r"(scale[k]));
+                }
+            }
+        }
+        if (SUMMED) {
+#pragma unroll
+            for (int i = 0; i < CH / 2; ++i) {
+                asm("dp2a.lo.u32.u32 %0, %1, %2, %0;" : "+r"(acc[2 * i]) : "r"(even[i]), "r"(scale[0]));
+                asm("dp2a.lo.u32.u32 %0, %1, %2, %0;" : "+r"(acc[2 * i]) : "r"(odd[i]), "r"(scale[1]));
+                asm("dp2a.hi.u32.u32 %0, %1, %2, %0;" : "+r"(acc[2 * i + 1]) : "r"(even[i]), "r"(scale[0]));
+                asm("dp2a.hi.u32.u32 %0, %1, %2, %0;" : "+r"(acc[2 * i + 1]) : "r"(odd[i]), "r"(scale[1]));
+            }
+        }
+        float o8[CH];
+        {
+            const float bs = base * sd, cs = bias * sd;
+#pragma unroll
+            for (int i = 0; i < CH; ++i) o8[i] = fmaf((float)acc[i], bs, cs);
+        }
+        if (fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
+            // too coarse for this deviation: the float32 codewords themselves, summed in stage order
+            float ex[CH];
+#pragma unroll
+            for (int i = 0; i < CH; ++i) ex[i] = 0.0f;
+            const uint32_t cn[4] = {n0, n1, n2, n3};
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                uint32_t j = (r & 1) ? (cn[r >> 1] >> 16) : (cn[r >> 1] & 0xFFFFu);
+                if (j >= Ku) j = 0;
+                const float4 *e = reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * 32 + slice * CH);
+#pragma unroll
+                for (int q = 0; q < CH / 4; ++q) {
+                    const float4 t = __ldg(e + q);
+                    ex[4 * q] += t.x; ex[4 * q + 1] += t.y; ex[4 * q + 2] += t.z; ex[4 * q + 3] += t.w;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < CH; ++i) o8[i] = ex[i] * sd;
+        }
+        uint32_t w[CH / 2];
+#pragma unroll
+        for (int c = 0; c < CH / 2; ++c) w[c] = Out<DT>::pack(o8[2 * c], o8[2 * c + 1]);
+        uint16_t *o16 = reinterpret_cast<uint16_t *>(out) + (size_t)v * stride;
+        if (LAYOUT == RVQ_GROUP_CONTIGUOUS) {
+            if (live) {
+                if (CH == 8)
+                    *reinterpret_cast<uint4 *>(o16 + g * 32 + slice * 8) = make_uint4(w[0], w[1], w[CH / 2 - 2], w[CH / 2 - 1]);
+                else
+                    *reinterpret_cast<uint2 *>(o16 + g * 32 + slice * 4) = make_uint2(w[0], w[1]);
+            }
+        } else if (CH == 8) {
+            // Lane g holds element pairs (2c, 2c+1) of group g, i.e. channels 32 slice + 8c + g and + 4.
+            // Lane c' of the 4-lane set wants pairs c' of all four groups: a 4x4 transpose of words in
+            // two butterfly steps (odd/even words with lane g^1, then word pairs with lane g^2).
+            uint32_t &w0 = w[0], &w1 = w[1], &w2 = w[CH / 2 - 2], &w3 = w[CH / 2 - 1];
+            const bool b1 = g & 1u, b2 = g & 2u;
+            const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w0 : w1, 1);
+            const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, b1 ? w2 : w3, 1);
+            if (b1) { w0 = r0; w2 = r1; } else { w1 = r0; w3 = r1; }
+            const uint32_t r2 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w0 : w2, 2);
+            const uint32_t r3 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w1 : w3, 2);
+            if (b2) { w0 = r2; w1 = r3; } else { w2 = r2; w3 = r3; }
+            // now w[q] = pair g of group q; channels 32 slice + 8 g + 0..7: element 2g of groups 0..3, then 2g+1
+            const uint32_t o0 = __byte_perm(w0, w1, 0x5410), o1 = __byte_perm(w2, w3, 0x5410);
+            const uint32_t o2 = __byte_perm(w0, w1, 0x7632), o3 = __byte_perm(w2, w3, 0x7632);
+            if (live) *reinterpret_cast<uint4 *>(o16 + slice * 32 + g * 8) = make_uint4(o0, o1, o2, o3);
+        } else {
+            // Lane g holds elements 4 slice + 0..3 of group g as w[0] = (e0, e1), w[1] = (e2, e3); the 16
+            // channels 16 slice .. 16 slice + 15 are element-major, so lane L stores element L of the four
+            // groups.  Exchange words with lane g^2, then halves with lane g^1.
+            const bool b1 = g & 1u, b2 = g & 2u;
+            const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w[0] : w[1], 2);
+            const uint32_t lo_g = b2 ? r0 : w[0], hi_g = b2 ? w[1] : r0;
+            const uint32_t keep = __byte_perm(lo_g, hi_g, b1 ? 0x7632 : 0x5410);
+            const uint32_t send = __byte_perm(lo_g, hi_g, b1 ? 0x5410 : 0x7632);
+            const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+            const uint32_t even = b1 ? got : keep, odd = b1 ? keep : got;
+            if (live)
+                *reinterpret_cast<uint2 *>(o16 + 4 * (slice * 4 + g)) =
+                    make_uint2(__byte_perm(even, odd, 0x5410), __byte_perm(even, odd, 0x7632));
+        }
+    }
+    if (bad && st && slice == 0) atomicAdd(&st->bad_codes, bad);   // every slice sees the same codes
+}
+
 // True when more than an eighth of a sample of up to 256 deviations is beyond the level tables' reach.
 // Uniform over the CTA (and over all CTAs of a launch: they read the same sample).
 __device__ __forceinline__ bool sample_wants_float32(const uint16_t *__restrict__ std16, int64_t n,
@@ -504,6 +729,40 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
     extern __shared__ __align__(128) uint8_t table[];
     if (PICK != 0 && sample_wants_float32(std16, n, dsec, 0.9e-3f) != (PICK == 2)) return;
     decode_sliced_body<DT, CH, F32T>(s, codes, std16, n, dsec, cb, out, stride, st, table);
+}
+
+// 0: summed-level tables, 1: per-stage scaled levels, 2: float32 tables -- the first kind within whose reach
+// at least seven eighths of a sample of up to 256 deviations lie.  Uniform over all CTAs of a launch.
+__device__ __forceinline__ int sample_table_kind(const uint16_t *__restrict__ std16, int64_t n, const uint8_t *__restrict__ dsec)
+{
+    const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
+    const float above_l = dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY;
+    const float above_s = dp->perr > 0.0f ? 0.9e-3f / dp->perr : INFINITY;
+    const int64_t samples = n < 256 ? n : 256, every = n < 256 ? 1 : n >> 8;
+    const float sd = threadIdx.x < samples ? fabsf(__half2float(__ushort_as_half(std16[threadIdx.x * every]))) : 0.0f;
+    const int far_s = __syncthreads_count(sd > above_s);
+    const int far_l = __syncthreads_count(sd > above_l);
+    if ((int64_t)far_s * 8 <= samples) return 0;
+    return (int64_t)far_l * 8 <= samples ? 1 : 2;
+}
+
+// One launch for the quoted shapes (dim 128, depth 8, 16-bit outputs, up to 3072 codes): every CTA
+// reads the same sample of deviations and takes the level tables (fast body) or, when the deviations
+// are beyond their reach, the float32 tables; both carve their slices out of whatever grid they get.
+template <int DT, int LCH, int FCH, int LAYOUT, int BITS>
+__global__ void __launch_bounds__(kDecThreads, 1)
+decode_quoted_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                     const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
+                     int64_t stride, rvq_status *st)
+{
+    extern __shared__ __align__(128) uint8_t table[];
+    const int kind = sample_table_kind(std16, n, dsec);
+    if (kind == 2)
+        decode_sliced_body<DT, FCH, true>(s, codes, std16, n, dsec, cb, out, stride, st, table);
+    else if (kind == 1)
+        decode_levels_fast<DT, LCH, LAYOUT, BITS, false>(s, codes, std16, n, dsec, cb, out, stride, st, table);
+    else
+        decode_levels_fast<DT, LCH, LAYOUT, BITS, true>(s, codes, std16, n, dsec, cb, out, stride, st, table);
 }
 
 // Decode with the rotary embedding, 4-channel slices (dim 128): float32 tables up to 1792 codes per stage,
@@ -683,6 +942,29 @@ int launch_decode_sliced(const Shape &s, const void *codes, const uint16_t *std1
         kernel<<<parts * ns, kDecThreads, smem, stream>>>(s, codes, std16, n, p + off, cb, out, stride, st);
         return check_launch();
     };
+    // the quoted shapes: one launch, tables chosen on the device
+    if (both && s.G == 4 && s.R == 8 && n * 4 < 0x7FFFFFFFLL && (s.bits == 16 || (s.bits >= 10 && s.bits <= 12)) &&
+        !(lch == 4 && fch == 4)) {
+        auto quoted = [&](auto kernel) -> int {
+            const size_t smem = (size_t)s.K * 16 * lch > (size_t)s.K * 32 * fch ? (size_t)s.K * 16 * lch : (size_t)s.K * 32 * fch;
+            int grid = sms < 8 ? 8 : sms;
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return RVQ_ERR_LAUNCH;
+            kernel<<<grid, kDecThreads, smem, stream>>>(s, codes, std16, n, p + off, cb, out, stride, st);
+            return check_launch();
+        };
+#define RVQ_Q4(DT, LCH, FCH, LAY)                                                                                   \
+        (s.bits == 16 ? quoted(decode_quoted_kernel<DT, LCH, FCH, LAY, 16>)                                          \
+         : s.bits == 10 ? quoted(decode_quoted_kernel<DT, LCH, FCH, LAY, 10>)                                        \
+         : s.bits == 11 ? quoted(decode_quoted_kernel<DT, LCH, FCH, LAY, 11>)                                        \
+                        : quoted(decode_quoted_kernel<DT, LCH, FCH, LAY, 12>))
+#define RVQ_Q3(DT, LAY) (lch == 8 ? RVQ_Q4(DT, 8, 4, LAY) : RVQ_Q4(DT, 4, 2, LAY))
+#define RVQ_Q2(DT) (s.layout == RVQ_GROUP_CONTIGUOUS ? RVQ_Q3(DT, RVQ_GROUP_CONTIGUOUS) : RVQ_Q3(DT, RVQ_GROUP_STRIDED))
+        return s.dtype == RVQ_BF16 ? RVQ_Q2(RVQ_BF16) : RVQ_Q2(RVQ_F16);
+#undef RVQ_Q2
+#undef RVQ_Q3
+#undef RVQ_Q4
+    }
 #define RVQ_DEC_F32(DT, PICK)                                                                                       \
     (fch == 4 ? launch(decode_sliced_kernel<DT, 4, true, PICK>, 4, true)                                           \
               : launch(decode_sliced_kernel<DT, 2, true, PICK>, 2, true))

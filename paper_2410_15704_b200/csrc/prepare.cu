@@ -32,7 +32,7 @@ static size_t decode_section_offset(const Shape &s)
 size_t prepared_bytes(const Shape &s)
 {
     size_t b = decode_section_offset(s);
-    if (decode_levels_prepared(s)) b += 256 + decode_table_bytes(s.K);
+    if (decode_levels_prepared(s)) b += 256 + 2 * decode_table_bytes(s.K);
     return (b + 255) / 256 * 256;
 }
 
@@ -68,12 +68,33 @@ decode_table_kernel(Shape s, const float *__restrict__ cb, const DecodeParams *_
         }
         w[c] = pair;
     }
+    // the same entry in units of its stage parity (summed levels)
+    uint32_t pw[4];
+    const float pst = r < 8 ? dp->pstep[r & 1] : 0.0f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint32_t pair = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t level = 0;
+            if (used && pst > 0.0f) {
+                const float q = rintf((v[2 * c + h] - lo[r]) / pst);
+                level = (uint32_t)fminf(fmaxf(q, 0.0f), 65535.0f);
+            }
+            pair |= level << (16 * h);
+        }
+        pw[c] = pair;
+    }
+    uint4 *ptable = table + decode_table_bytes(s.K) / sizeof(uint4);
     if (wide) {
         table[((size_t)octet * s.K + j) * 8 + r] = make_uint4(w[0], w[1], w[2], w[3]);
+        ptable[((size_t)octet * s.K + j) * 8 + r] = make_uint4(pw[0], pw[1], pw[2], pw[3]);
     } else {
-        uint2 *t2 = reinterpret_cast<uint2 *>(table);
+        uint2 *t2 = reinterpret_cast<uint2 *>(table), *p2 = reinterpret_cast<uint2 *>(ptable);
         t2[((size_t)(2 * octet) * s.K + j) * 8 + r] = make_uint2(w[0], w[1]);
         t2[((size_t)(2 * octet + 1) * s.K + j) * 8 + r] = make_uint2(w[2], w[3]);
+        p2[((size_t)(2 * octet) * s.K + j) * 8 + r] = make_uint2(pw[0], pw[1]);
+        p2[((size_t)(2 * octet + 1) * s.K + j) * 8 + r] = make_uint2(pw[2], pw[3]);
     }
 }
 
@@ -166,6 +187,31 @@ prepare_params_kernel(Shape s, const StagePartial *__restrict__ part, PreparedHe
                 b += s_lo[q]; e += 0.5f * (float)sc * base * 1.0001f;             // half a level per stage
             }
             dp->bias = b; dp->err = e; dp->base = base;
+            // summed levels: per parity the finest unit such that the four stages' top levels add up to
+            // at most 65535 (each stage's top level is its range over the unit, rounded up: 8 spare levels),
+            // expressed as an integer multiple (1..255) of a base of their own
+            float punit[2] = {0.0f, 0.0f}, pe = 0.0f;
+            int pstages[2] = {0, 0};
+            for (int par = 0; par < 2; ++par) {
+                float span = 0.0f;
+                for (int q = par; q < 8; q += 2)
+                    if (s_step[q] > 0.0f) { span += s_step[q] * 65535.0f; ++pstages[par]; }
+                punit[par] = span / (65535.0f - 8.0f);
+            }
+            const float pbase = fmaxf(punit[0], punit[1]) * 1.000001f / 255.0f;
+            for (int par = 0; par < 2; ++par) {
+                uint32_t sc = 0;
+                if (pstages[par] > 0 && pbase > 0.0f) {
+                    sc = (uint32_t)fminf(255.0f, ceilf(punit[par] / pbase));
+                    while (sc < 255u && (float)sc * pbase < punit[par]) ++sc;
+                    if (!((float)sc * pbase >= punit[par])) pe = INFINITY;     // (rounding at 255: no summed tables)
+                }
+                dp->pscale[par] = sc;
+                dp->pstep[par] = (float)sc * pbase;
+                pe += 0.5f * (float)pstages[par] * (float)sc * pbase * 1.0001f;   // half a level per stage
+            }
+            dp->pbase = pbase;
+            dp->perr = pe;
         }
     }
 }

@@ -36,11 +36,20 @@ struct DecodeParams {
     float base;
     float pad[5];
     uint32_t scale[8]; // integer scale of a stage's levels (0 for absent stages)
+    // Second set of tables ("summed levels"): the stages of one parity (even r, odd r) share a unit
+    // fine enough that the levels of all four of them add up to at most 65535, so a decoder adds
+    // table words as they are (two 16-bit fields per 32-bit word, no carry between them) and scales
+    // once per parity.  Coarser than the tables above by a factor of about four.
+    float pstep[2];      // value of one summed level, pscale * pbase, for even / odd stages; 0 if unused
+    float perr;          // bound on |sum of summed-table values - sum of float32 values| per channel
+    float pbase;         // common base of the two parities' units
+    uint32_t pscale[2];  // integer scales (1..255) of the two parities
 };
 constexpr int kDecodeWideK = 1536;                        // 128 bytes per code per slice in shared memory
 constexpr int kDecodeMaxK = 3072;                         // 64 bytes per code per slice
 __host__ __device__ inline int decode_slice_channels(int K) { return K <= kDecodeWideK ? 8 : 4; }
 __host__ __device__ inline size_t decode_table_bytes(int K) { return (size_t)K * 512; }   // 32 channels x 8 stages x 2 bytes
+// the prepared block holds two such tables: levels scaled per stage, then levels summed per stage parity
 constexpr int kDecodeExactWideK = 1792;                   // float32 tables: 128 bytes per code per 4-channel slice
 constexpr int kDecodeExactK = 3584;                       // ... 64 bytes per code per 2-channel slice
 // Which decoder serves a shape (group_dim 32, a power-of-two number of groups up to 32, depth <= 8; everything

@@ -62,6 +62,134 @@ ema_stats_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t stride,
     }
 }
 
+// Groups of 32 channels, at most 8 groups and 32 codes per head vector: one warp per head vector, lane = channel
+// of the group.  A row's 32 floats then go to their bin as one coalesced 128-byte reduction (four
+// sectors, one cache line) and the codeword that takes the residual to the next stage comes in as one
+// 128-byte load, where a thread per row would scatter both over 32 lines per instruction (the L1's tag
+// stage, not the atomics in L2, was what bound that form).  Counts go to a histogram [R][K] in shared
+// memory, lanes that share a bin adding once (match.any), merged into the global counts once per CTA.
+constexpr int kWarpStatsThreads = 256;
+
+__global__ void __launch_bounds__(kWarpStatsThreads)
+ema_stats_warp_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t stride,
+                      const void *__restrict__ codes, const float *__restrict__ cb,
+                      uint32_t *__restrict__ cnt, float *__restrict__ sum, rvq_status *st)
+{
+    extern __shared__ uint32_t hist[];                       // [R][K]
+    const int bins = s.R * s.K;
+    for (int t = threadIdx.x; t < bins; t += kWarpStatsThreads) hist[t] = 0u;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int warps = (kWarpStatsThreads / 32) * gridDim.x;
+    const int G = s.G, R = s.R, per = s.per_vector;            // per = G * R <= 32
+    uint32_t bad = 0;
+    for (int64_t v = (int64_t)blockIdx.x * (kWarpStatsThreads / 32) + warp; v < n; v += warps) {
+        // element `lane` of every group: channel g*32+lane (contiguous groups) or lane*G+g (strided)
+        float z[8];                                            // (G <= 8)
+        float a = 0.0f;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            z[g] = g < G ? load_as_float(x, v * stride + channel_of(s.layout, G, 32, g, lane), s.dtype) : 0.0f;
+            a += z[g];
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xFFFFFFFFu, a, off);
+        const float mu = a / (float)s.dim;
+        float b = 0.0f;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) b += g < G ? (z[g] - mu) * (z[g] - mu) : 0.0f;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, off);
+        const float dev = sqrtf(b / (float)(s.dim - s.ddof));
+        const bool deg = deviation_is_degenerate(dev);
+        // lane l holds code l of the vector (group l / R, stage l % R) and counts it
+        uint32_t code = 0;
+        if (lane < per) {
+            code = read_code(reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes, lane, s.bits, s.code_bytes);
+            if (code >= (uint32_t)s.K) { code = 0; ++bad; }
+        }
+        const int my_bin = lane < per ? (lane % R) * s.K + (int)code : -1 - lane;   // (idle lanes: bins of their own)
+        const uint32_t same = __match_any_sync(0xFFFFFFFFu, my_bin);
+        if (lane < per && lane == __ffs(same) - 1) atomicAdd(&hist[my_bin], (uint32_t)__popc(same));
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            if (g >= G) break;
+            float zr = deg ? 0.0f : z[g] / dev;
+            for (int r = 0; r < R; ++r) {
+                const uint32_t j = __shfl_sync(0xFFFFFFFFu, code, g * R + r);
+                const size_t at = ((size_t)r * s.K + j) * 32 + lane;
+                const float e = __ldg(cb + at);
+                atomicAdd(sum + at, zr);
+                zr -= e;
+            }
+        }
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < bins; t += kWarpStatsThreads)
+        if (hist[t]) atomicAdd(cnt + t, hist[t]);
+    if (bad && st && lane < 32) atomicAdd(&st->bad_codes, bad);
+}
+
+// The same for head vectors of exactly four groups (dim 128): the warp takes the four rows of a vector
+// at once, lane = (group, four-channel piece), so that every stage is one 16-byte reduction and one
+// 16-byte load per lane (four cache lines per instruction) instead of eight instructions per row.
+__global__ void __launch_bounds__(kWarpStatsThreads)
+ema_stats_quad_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t stride,
+                      const void *__restrict__ codes, const float *__restrict__ cb,
+                      uint32_t *__restrict__ cnt, float *__restrict__ sum, rvq_status *st)
+{
+    extern __shared__ uint32_t hist[];                       // [R][K]
+    const int bins = s.R * s.K;
+    for (int t = threadIdx.x; t < bins; t += kWarpStatsThreads) hist[t] = 0u;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int warps = (kWarpStatsThreads / 32) * gridDim.x;
+    const int R = s.R, per = s.per_vector;                     // per = 4 * R <= 32
+    const int g = lane >> 3, q = lane & 7;                     // this lane: elements 4q .. 4q+3 of group g
+    uint32_t bad = 0;
+    for (int64_t v = (int64_t)blockIdx.x * (kWarpStatsThreads / 32) + warp; v < n; v += warps) {
+        float z[4];
+        float a = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            z[k] = load_as_float(x, v * stride + channel_of(s.layout, 4, 32, g, 4 * q + k), s.dtype);
+            a += z[k];
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xFFFFFFFFu, a, off);
+        const float mu = a / (float)s.dim;
+        float b = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) b += (z[k] - mu) * (z[k] - mu);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, off);
+        const float dev = sqrtf(b / (float)(s.dim - s.ddof));
+        const bool deg = deviation_is_degenerate(dev);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) z[k] = deg ? 0.0f : z[k] / dev;
+        // lane l holds code l of the vector (group l / R, stage l % R) and counts it
+        uint32_t code = 0;
+        if (lane < per) {
+            code = read_code(reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes, lane, s.bits, s.code_bytes);
+            if (code >= (uint32_t)s.K) { code = 0; ++bad; }
+        }
+        const int my_bin = lane < per ? (lane % R) * s.K + (int)code : -1 - lane;   // (idle lanes: bins of their own)
+        const uint32_t same = __match_any_sync(0xFFFFFFFFu, my_bin);
+        if (lane < per && lane == __ffs(same) - 1) atomicAdd(&hist[my_bin], (uint32_t)__popc(same));
+        for (int r = 0; r < R; ++r) {
+            const uint32_t j = __shfl_sync(0xFFFFFFFFu, code, g * R + r);
+            const size_t at = ((size_t)r * s.K + j) * 32 + 4 * q;
+            const float4 e = __ldg(reinterpret_cast<const float4 *>(cb + at));
+            atomicAdd(reinterpret_cast<float4 *>(sum + at), make_float4(z[0], z[1], z[2], z[3]));
+            z[0] -= e.x; z[1] -= e.y; z[2] -= e.z; z[3] -= e.w;
+        }
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < bins; t += kWarpStatsThreads)
+        if (hist[t]) atomicAdd(cnt + t, hist[t]);
+    if (bad && st) atomicAdd(&st->bad_codes, bad);
+}
+
 __global__ void __launch_bounds__(256)
 counts_to_float_kernel(const uint32_t *__restrict__ cnt, float *__restrict__ out, int total)
 {
@@ -129,7 +257,23 @@ int launch_ema_stats(const Shape &s, const void *x, int64_t n, int64_t stride, c
         cudaMemsetAsync(batch_sum, 0, (size_t)bins * s.gd * sizeof(float), stream) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
     int rc = RVQ_OK;
-    if (n > 0) {
+    if (n > 0 && s.gd == 32 && s.G <= 8 && s.per_vector <= 32 && (size_t)bins * sizeof(uint32_t) <= 160 * 1024) {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return RVQ_ERR_DEVICE;
+        const size_t smem = (size_t)bins * sizeof(uint32_t);
+        // as many CTAs per SM as the histograms leave room for (up to 8 of 256 threads)
+        int per_sm = (int)((200 * 1024) / (smem + 1024));
+        per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+        int64_t want = (n + kWarpStatsThreads / 32 - 1) / (kWarpStatsThreads / 32);
+        int grid = (int)(want < (int64_t)sms * per_sm ? want : (int64_t)sms * per_sm);
+        auto kernel = s.G == 4 ? ema_stats_quad_kernel : ema_stats_warp_kernel;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return RVQ_ERR_LAUNCH;
+        kernel<<<grid, kWarpStatsThreads, smem, stream>>>(s, x, n, stride, codes, cb, cnt, batch_sum, st);
+        rc = check_launch();
+    } else if (n > 0) {
         switch (s.gd) {
         case 8: rc = stats_gd<8>(s, x, n, stride, codes, cb, cnt, batch_sum, st, stream); break;
         case 16: rc = stats_gd<16>(s, x, n, stride, codes, cb, cnt, batch_sum, st, stream); break;

@@ -334,8 +334,10 @@ int rvq_kmeans_init(const rvq_config *cfg /* host */, const void *x, int64_t n, 
  *
  * Arguments, results and error codes are those of rvq_ema_update.  Differences:
  *   - The first call on each device looks up the array's device address (a
- *     runtime query, not a launch).  Make that first call outside any stream
- *     capture.
+ *     runtime query, not a launch) and keeps it.  Make that first call outside
+ *     any stream capture.  The kept address belongs to the device's primary
+ *     context: after cudaDeviceReset the array lives elsewhere, so do not call
+ *     this entry point on a device that has been reset since its first call.
  *   - All calls, on every stream, share the one array, and it still holds the
  *     previous call's numbers when the next begins; each call clears the parts
  *     it accumulates into.  Two calls that can overlap on the GPU (different

@@ -53,7 +53,7 @@ NEAR_TIE = 1e-5
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (OpenMP over head vectors)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+        subprocess.check_call(["gcc", "-O3", "-fopenmp", "-fPIC", "-shared", "-std=c11",
                                "-o", _LIB, _SRC, "-lm"])
     return _LIB
 

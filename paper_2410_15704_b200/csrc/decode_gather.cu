@@ -42,7 +42,11 @@ int launch_decode_gather(const Shape &s, const void *codes, const uint16_t *std1
     if (n == 0) return RVQ_OK;
     const int64_t total = n * s.G * (s.gd / 4);
     int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 64) blocks = 148 * 64;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return RVQ_ERR_DEVICE;
+    if (blocks > (int64_t)sms * 64) blocks = (int64_t)sms * 64;
     decode_gather_kernel<<<(unsigned)blocks, 256, 0, stream>>>(s, codes, std16, n, cb, out, stride, st);
     return check_launch();
 }

@@ -862,7 +862,11 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
         int vpb = 256 / per_vec;
         if (vpb < 1) vpb = 1;
         int64_t blocks = (n + vpb - 1) / vpb;
-        if (blocks > 148 * 16) blocks = 148 * 16;
+        int dev_g = 0, sms_g = 0;
+        if (cudaGetDevice(&dev_g) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms_g, cudaDevAttrMultiProcessorCount, dev_g) != cudaSuccess)
+            return RVQ_ERR_DEVICE;
+        if (blocks > (int64_t)sms_g * 16) blocks = (int64_t)sms_g * 16;
         const size_t smem = (size_t)vpb * s.dim * sizeof(float);
         decode_rope_gather_kernel<<<(unsigned)blocks, 256, smem, stream>>>(s, codes, std16, n, cb, out, stride, st, ra,
                                                                            style == 0 ? 1 : 2, vpb);

@@ -3,6 +3,8 @@
 // normalisation.
 #include "common.cuh"
 
+#include <atomic>
+
 namespace rvq {
 
 static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
@@ -324,7 +326,11 @@ constexpr size_t kStaticScratchBytes = 65536 + 65536 + 2097152;
 static __device__ __align__(256) unsigned char g_ema_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void *g_scratch_addr[kMaxDevices];      // device address of g_ema_scratch per device ordinal (null: not looked up yet)
+// Device address of g_ema_scratch per device ordinal (null: not looked up yet).  Host threads may race to
+// fill an entry: they all store the same value, and the atomic keeps the store and the loads whole.  The
+// cache assumes the runtime's one primary context per device; after cudaDeviceReset the array lives at a
+// new address, so a process that resets a device must not call this entry point on it again.
+std::atomic<void *> g_scratch_addr[kMaxDevices];
 
 // The array's name is only a handle on the host; the address a kernel can use
 // has to be asked for, once per device, with that device current.
@@ -332,12 +338,12 @@ int static_scratch(void **out)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RVQ_ERR_DEVICE;
-    if (!g_scratch_addr[dev]) {
-        void *ptr = nullptr;
+    void *ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress(&ptr, g_ema_scratch) != cudaSuccess || !ptr) return RVQ_ERR_DEVICE;
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = ptr;
     return RVQ_OK;
 }
 

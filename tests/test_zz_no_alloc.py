@@ -42,9 +42,13 @@ def test_static_scratch_update_matches_workspace_update_twice():
         state["sta"]["n"].copy_(state["ref"]["n"]); state["sta"]["m"].copy_(state["ref"]["m"])
         rvq.rvq_ema_update(cfg, x, w.n, w.dim, ref.codes, ref.codebooks, state["ref"]["n"], state["ref"]["m"],
                            state["ref"]["batch"], w.decay, w.eps, ref.workspace, ref.workspace_bytes, ref.status)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         rvq.rvq_ema_update_static(cfg, x, w.n, w.dim, ref.codes, sta.codebooks, state["sta"]["n"],
                                   state["sta"]["m"], state["sta"]["batch"], w.decay, w.eps, sta.status)
         torch.cuda.synchronize()
+        # the call took no device memory (torch's allocator was not involved either: the binding passes pointers)
+        assert torch.cuda.mem_get_info()[0] == free_before
         assert torch.equal(state["ref"]["batch"], state["sta"]["batch"])              # counts are integers
         assert int(state["sta"]["batch"].sum().item()) == w.n * w.groups * R
         assert torch.max(torch.abs(ref.codebooks - sta.codebooks)).item() <= TOL

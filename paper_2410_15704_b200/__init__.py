@@ -56,6 +56,8 @@ def _load() -> ctypes.CDLL:
     lib.rvq_prepare_codebooks.argtypes = [cfgp, vp, vp, vp]
     lib.rvq_encode.restype = ctypes.c_int
     lib.rvq_encode.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.rvq_selftest_encode_timeout.restype = ctypes.c_int
+    lib.rvq_selftest_encode_timeout.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, ctypes.c_uint32, vp, vp]
     lib.rvq_encode_exact.restype = ctypes.c_int
     lib.rvq_encode_exact.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp]
     lib.rvq_encode_stats.restype = ctypes.c_int
@@ -91,7 +93,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 
-EXPORTS = ("rvq_rope_table", "rvq_decode_rope", "rvq_learn_step", "rvq_kmeans_workspace_bytes", "rvq_kmeans_init", "rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
+EXPORTS = ("rvq_selftest_encode_timeout", "rvq_rope_table", "rvq_decode_rope", "rvq_learn_step", "rvq_kmeans_workspace_bytes", "rvq_kmeans_init", "rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
            "rvq_prepare_codebooks", "rvq_workspace_bytes", "rvq_encode", "rvq_decode",
            "rvq_ema_update")
 
@@ -164,6 +166,16 @@ def rvq_encode_stats(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f1
                               _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_encode_stats")
+    return rc
+
+
+def rvq_selftest_encode_timeout(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, wait_polls, status,
+                                stream=None, check=True) -> int:
+    """rvq_encode with one MMA chain left out per CTA: its wait gives up (include/rvq_selftest.h)."""
+    rc = lib.rvq_selftest_encode_timeout(ctypes.byref(cfg), _ptr(x), n, x_row_stride, _ptr(codebooks), _ptr(prepared),
+                                         _ptr(codes), _ptr(std_f16), wait_polls, _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_selftest_encode_timeout")
     return rc
 
 

@@ -3,6 +3,7 @@
 // state: the launch counter below, and (in ema.cu) the per-device address of
 // the built-in scratch array of rvq_ema_update_static.
 #include "prepared.cuh"
+#include "rvq_selftest.h"
 
 #include <atomic>
 
@@ -162,6 +163,21 @@ int rvq_encode_stats(const rvq_config *cfg, const void *x, int64_t n, int64_t x_
                        cnt, batch_sum);
     if (rc != RVQ_OK) return rc;
     return launch_counts_to_float(cnt, batch_count, bins, st);
+}
+
+int rvq_selftest_encode_timeout(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,
+                                const float *codebooks, const void *prepared, void *codes, uint16_t *std_f16,
+                                uint32_t wait_polls, rvq_status *status, void *stream)
+{
+    Shape s;
+    int rc = make_shape(cfg, &s);
+    if (rc != RVQ_OK) return rc;
+    if ((rc = check_rows(s, x, n, x_row_stride)) != RVQ_OK) return rc;
+    if (!codebooks || !prepared || !status || (n > 0 && (!codes || !std_f16))) return RVQ_ERR_BADARG;
+    if (!aligned16(codebooks) || !aligned16(codes) || !aligned256(prepared)) return RVQ_ERR_ALIGN;
+    if (!encode_tensor_supported(s) || wait_polls < 1024u) return RVQ_ERR_UNSUPPORTED;
+    return launch_encode_tensor(s, x, n, x_row_stride, codebooks, prepared, codes, std_f16, status,
+                                (cudaStream_t)stream, nullptr, nullptr, nullptr, wait_polls, 1);
 }
 
 int rvq_encode_exact(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,

@@ -34,7 +34,7 @@ bool encode_tensor_supported(const Shape &s);
 int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
                          const void *prepared, void *codes, uint16_t *std16, rvq_status *st,
                          cudaStream_t stream, uint32_t *stat_cnt = nullptr, float *stat_sum = nullptr,
-                         float *energy = nullptr);
+                         float *energy = nullptr, uint32_t wait_limit = 0, int drop_last_chain = 0);
 int launch_counts_to_float(const uint32_t *cnt, float *out, int bins, cudaStream_t stream);
 int launch_decode_gather(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
                          const float *cb, void *out, int64_t stride, rvq_status *st,

@@ -76,7 +76,8 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 // Bounded wait; returns false (and raises the CTA's abort flag) when it gives up.  A phase that has
 // completed already is recognised by the non-blocking test (a plain shared-memory read); only a
 // phase still pending goes through the suspending form.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          uint32_t limit = kWaitLimit)
 {
     uint32_t ok;
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -84,7 +85,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     if (ok) return true;
 #pragma unroll 1
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
                      "selp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
@@ -285,6 +286,8 @@ struct Params {
     uint32_t *stat_cnt; // optional EMA statistics of this batch: counts [R][K] ...
     float *stat_sum;    // ... and sums of the stage inputs [R][K][32]; both null when not wanted
     float *energy;      // optional [R]: sum over the rows of the squared norm of what each stage leaves
+    uint32_t wait_limit;   // polls after which a wait gives up (kWaitLimit; smaller only in the timeout self-test)
+    int drop_last_chain;   // timeout self-test: 1 = tile 0's issuer leaves out the CTA's very last chain; else 0
 };
 
 // The tiles of one CTA: a contiguous run, done in `rounds` rounds of nearly equal size (<= kTiles).
@@ -404,6 +407,9 @@ encode_tensor_kernel(const Params p)
                 first = false;
                 tc_fence_after();
                 const uint64_t bd = bdesc0 + (uint64_t)(slot * (uint32_t)(kSlotBytes >> 4));
+                // (self-test of the give-up path: the chain that nothing comes after is left out, so that the
+                // epilogue's wait for it runs out with no copy or MMA of this CTA still in flight)
+                if (p.drop_last_chain && t == 0 && q == total - 1) break;
                 mma_f16_ts(acc, a0, bd, idesc, 0);                      // hi[0:16]  . hi cells 0-1
                 mma_f16_ts(acc, a0 + 8, bd + 2 * 128, idesc, 1);        // hi[16:32] . hi cells 2-3
                 mma_f16_ts(acc, a0, bd + 4 * 128, idesc, 1);            // hi[0:16]  . lo cells 4-5
@@ -571,7 +577,7 @@ encode_tensor_kernel(const Params p)
                         const int pj = min(pb * 128 + pbb * 32 + 3 * pq + pk, s.K - 1);
                         asm volatile("prefetch.global.L1 [%0];" ::"l"(cbr + (size_t)pj * 32));
                     }
-                    ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag);
+                    ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag, p.wait_limit);
                     ok = __all_sync(0xFFFFFFFFu, ok);          // tcgen05.ld below needs the whole warp
                     ++chunk_use;
                     if (!ok) break;
@@ -788,7 +794,8 @@ bool encode_tensor_supported(const Shape &s)
 
 int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
                          const void *prepared, void *codes, uint16_t *std16, rvq_status *st,
-                         cudaStream_t stream, uint32_t *stat_cnt, float *stat_sum, float *energy)
+                         cudaStream_t stream, uint32_t *stat_cnt, float *stat_sum, float *energy,
+                         uint32_t wait_limit, int drop_last_chain)
 {
     if (n == 0) return RVQ_OK;
     const int64_t rows = n * s.G;
@@ -801,7 +808,7 @@ int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t strid
     if (cudaFuncSetAttribute(encode_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
     Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)tiles, stat_cnt, stat_sum,
-             energy};
+             energy, wait_limit ? wait_limit : kWaitLimit, drop_last_chain};
     const int64_t groups = (tiles + kTiles - 1) / kTiles;
     const int grid = (int)(groups < sms ? groups : sms);
     encode_tensor_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);

@@ -471,6 +471,23 @@ def test_degenerate_vectors_and_bad_codes():
     assert_recon_match(got, fixed, std_bits, w.codebooks, w.dim, w.layout, cfg.x_dtype)
 
 
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """The encoder's bounded waits: with one MMA chain per CTA left out on purpose (nothing else in
+    flight behind it) the epilogue's wait gives up after 2^16 polls, the kernel returns, the status
+    block says so, and the next regular encode on the same context is exact."""
+    w = rvq_synth.key_cache(tokens=4096)
+    cfg = config_of(w)
+    xd = x_to_device(w.x, cfg.x_dtype)
+    b = rvq.alloc_buffers(cfg, w.n, w.codebooks)
+    rvq.rvq_selftest_encode_timeout(cfg, xd, w.n, w.dim, b.codebooks, b.prepared, b.codes, b.std, 1 << 16, b.status)
+    torch.cuda.synchronize()
+    st = rvq.read_status(b.status)
+    assert st["wait_timeouts"] >= 1
+    codes, std_bits, st2, _ = gpu_encode(cfg, xd, w.n, w.codebooks)
+    assert st2["wait_timeouts"] == 0
+    assert_codes_match(w.x, codes, w.codebooks, w.layout)
+
+
 def test_scale_invariance_on_gpu():
     w = rvq_synth.tiny(256)
     cfg = config_of(w)

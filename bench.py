@@ -258,7 +258,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     import paper_2410_15704_b200 as rvq
-    from paper_2410_15704_b200.dist import allreduce_stats
+    from paper_2410_15704_b200.dist import allreduce_stats, stats_buffer
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -283,8 +283,7 @@ def run_ours(args):
     recon = torch.empty(n, w.dim, dtype=torch.bfloat16, device="cuda")
     ema_count = torch.ones(R, K, device="cuda")
     ema_sum = b.codebooks.clone()
-    stats = torch.empty(R * K * (gd + 1), device="cuda")      # batch counts then batch sums, one all-reduce
-    bcount, bsum = stats[:R * K], stats[R * K:]
+    stats, bcount, bsum = stats_buffer(R, K, gd, "cuda")      # batch counts then batch sums, one all-reduce
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     codes_host = torch.empty_like(b.codes, device="cpu").pin_memory()
     std_host = torch.empty_like(b.std, device="cpu").pin_memory()

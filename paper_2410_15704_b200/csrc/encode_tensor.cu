@@ -184,41 +184,40 @@ struct Sweep {
     float zz;                // squared norm of the scaled residual: m1 + zz is the best squared distance
     int cnt;                 // listed chunks (kListCap + 1: the list overflowed)
     float bb[4];             // minimum per 32-column block position inside its 128-column chunk
-    float d[11];             // minimum per cell position (3 columns each, the last one 2)
-    float k[3];              // minimum per column position inside its cell
+    float h[2];              // minimum per half (columns 0-15, 16-31) of a block
+    float d[16];             // minimum per column position inside its half
 };
 
-// One 32-column block of scores (block `b` of its chunk): folds its eleven 3-column cell minima into
-// w.d, the minima of the three in-cell column positions into w.k and the block minimum into w.bb[b];
-// returns the block minimum.  A column that could be the argmin is thereby pinned to
-// (listed chunk) x (block of the chunk) x (cell position) x (position in the cell).
+// One 32-column block of scores (block `b` of its chunk) folded into the running minima of three
+// partitions of its columns: the 16 places inside a half (one three-input minimum takes in the two
+// columns of a place), the two halves, and the block itself; returns the block minimum.  Together
+// with the chunk list a column that could be the argmin is pinned to (listed chunk) x (block of the
+// chunk) x (half) x (place): when every one of the four lists has a single entry, to one column.
+// 36 minimum operations per 32 scores: they run on the narrow integer/compare pipe, which this sweep
+// keeps about as busy as the tensor pipe, so their number per score is what the sweep's speed
+// hangs on.
 __device__ __forceinline__ float fold_block(Sweep &w, const uint32_t (&u)[32], int b)
 {
-    float t[11];
 #pragma unroll
-    for (int q = 0; q < 10; ++q)
-        t[q] = min3(__uint_as_float(u[3 * q]), __uint_as_float(u[3 * q + 1]), __uint_as_float(u[3 * q + 2]));
-    t[10] = fminf(__uint_as_float(u[30]), __uint_as_float(u[31]));
+    for (int c = 0; c < 16; ++c) w.d[c] = min3(w.d[c], __uint_as_float(u[c]), __uint_as_float(u[c + 16]));
+    float hm[2];
 #pragma unroll
-    for (int q = 0; q < 11; ++q) w.d[q] = fminf(w.d[q], t[q]);
-#pragma unroll
-    for (int c = 0; c < 3; ++c) {
-        float m = w.k[c];
-#pragma unroll
-        for (int q = 0; q < 10; q += 2)
-            m = min3(m, __uint_as_float(u[3 * q + c]), __uint_as_float(u[3 * q + 3 + c]));
-        if (c < 2) m = fminf(m, __uint_as_float(u[30 + c]));      // the last cell has two columns
-        w.k[c] = m;
+    for (int hf = 0; hf < 2; ++hf) {
+        const uint32_t *v = u + 16 * hf;
+        const float a0 = min3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+        const float a1 = min3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+        const float a2 = min3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
+        const float a3 = min3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
+        const float a4 = min3(__uint_as_float(v[12]), __uint_as_float(v[13]), __uint_as_float(v[14]));
+        hm[hf] = fminf(min3(a0, a1, a2), min3(a3, a4, __uint_as_float(v[15])));
     }
-    const float m = min3(min3(min3(t[0], t[1], t[2]), min3(t[3], t[4], t[5]), min3(t[6], t[7], t[8])), t[9], t[10]);
+    w.h[0] = fminf(w.h[0], hm[0]);
+    w.h[1] = fminf(w.h[1], hm[1]);
+    const float m = fminf(hm[0], hm[1]);
     w.bb[b] = fminf(w.bb[b], m);
     return m;
 }
 
-// Keep a chunk's minimum if it is within the window of the running minimum.
-// Branch-free: the value is always written to the next free slot and the slot
-// is claimed only when it belongs on the list; slot kListCap is scratch once
-// the list has overflowed.
 // A column can only be the exact-L2 choice (in real arithmetic, and in the float32 direct-form
 // arithmetic of the all-float32 kernel, whose relative error on a distance is below 34 * 2^-24) if its
 // approximate score is at most threshold(m1): the window covers the approximation error of both
@@ -552,8 +551,8 @@ encode_tensor_kernel(const Params p)
                 w.zz = zz;
                 w.m1 = INFINITY; w.thr = INFINITY; w.cnt = 0;
 #pragma unroll
-                for (int q = 0; q < 11; ++q) w.d[q] = INFINITY;
-                w.k[0] = w.k[1] = w.k[2] = INFINITY;
+                for (int q = 0; q < 16; ++q) w.d[q] = INFINITY;
+                w.h[0] = w.h[1] = INFINITY;
                 w.bb[0] = w.bb[1] = w.bb[2] = w.bb[3] = INFINITY;
                 const bool force_scan = !(zmax < 60000.0f) || !(w.win < INFINITY);
 
@@ -562,19 +561,18 @@ encode_tensor_kernel(const Params p)
                     if (c == S - 1 && w.cnt > 0) {
                         // Before the last chunk the running winner is the final one most of the time:
                         // start fetching its codeword while the MMA chain runs.
-                        int pb = 0, pq = 0, pk = 0, pbb = 0;
+                        int pb = 0, pq = 0, ph = 0, pbb = 0;
 #pragma unroll
                         for (int e = kListCap - 1; e >= 0; --e)
                             if (e < w.cnt && list_v[e * kRowsPerPass] == w.m1) pb = list_i[e * kRowsPerPass];
 #pragma unroll
-                        for (int q = 10; q >= 0; --q)
+                        for (int q = 15; q >= 0; --q)
                             if (w.d[q] == w.m1) pq = q;
-                        if (w.k[1] == w.m1) pk = 1;
-                        if (w.k[2] == w.m1) pk = 2;
+                        if (w.h[1] == w.m1 && w.h[0] != w.m1) ph = 1;
 #pragma unroll
                         for (int i = 3; i > 0; --i)
                             if (w.bb[i] == w.m1) pbb = i;
-                        const int pj = min(pb * 128 + pbb * 32 + 3 * pq + pk, s.K - 1);
+                        const int pj = min(pb * 128 + pbb * 32 + 16 * ph + pq, s.K - 1);
                         asm volatile("prefetch.global.L1 [%0];" ::"l"(cbr + (size_t)pj * 32));
                     }
                     ok = mbar_wait(BAR(kBarAccFull + tile), chunk_use & 1u, abort_flag, p.wait_limit);
@@ -607,8 +605,8 @@ encode_tensor_kernel(const Params p)
                 const int cnt = w.cnt;
 
                 // ---- stage end: the columns that can still be the exact argmin are those of a listed
-                // block, at a listed cell position, at a listed place inside the cell.  When each of the
-                // three lists has one entry (almost always) that column is the choice: every other
+                // chunk, in a listed block of the chunk, in a listed half, at a listed place.  When each of
+                // the four lists has one entry (almost always) that column is the choice: every other
                 // column is farther than the approximation and float32 evaluation errors can bridge.
                 const float lim = threshold(w, m1);
                 int b1 = 0, nlisted = 0;
@@ -623,27 +621,27 @@ encode_tensor_kernel(const Params p)
                         if (live && !found && fv == m1) { found = true; b1 = fi; }
                     }
                 }
-                uint32_t qmask = 0u, kmask = 0u, bmask = 0u;
-                int q1 = 0, k1 = 0, bb1 = 0;
+                uint32_t qmask = 0u, hmask = 0u, bmask = 0u;
+                int q1 = 0, h1 = 0, bb1 = 0;
 #pragma unroll
                 for (int i = 3; i >= 0; --i) {
                     if (w.bb[i] <= lim) bmask |= 1u << i;
                     if (w.bb[i] == m1) bb1 = i;
                 }
 #pragma unroll
-                for (int q = 10; q >= 0; --q) {
+                for (int q = 15; q >= 0; --q) {
                     if (w.d[q] <= lim) qmask |= 1u << q;
                     if (w.d[q] == m1) q1 = q;
                 }
 #pragma unroll
-                for (int c = 2; c >= 0; --c) {
-                    if (w.k[c] <= lim) kmask |= 1u << c;
-                    if (w.k[c] == m1) k1 = c;
+                for (int c = 1; c >= 0; --c) {
+                    if (w.h[c] <= lim) hmask |= 1u << c;
+                    if (w.h[c] == m1) h1 = c;
                 }
-                const int j1 = b1 * 128 + bb1 * 32 + 3 * q1 + k1;
+                const int j1 = b1 * 128 + bb1 * 32 + 16 * h1 + q1;
                 // (a padded column scores 60000: if nothing real scored less, scan everything)
                 const bool scan_all = force_scan || cnt == 0 || cnt > kListCap || !(m1 < 59000.0f);
-                const bool unique = nlisted == 1 && (qmask & (qmask - 1u)) == 0u && (kmask & (kmask - 1u)) == 0u &&
+                const bool unique = nlisted == 1 && (qmask & (qmask - 1u)) == 0u && (hmask & (hmask - 1u)) == 0u &&
                                     (bmask & (bmask - 1u)) == 0u && j1 < s.K;
                 const bool flagged = !deg && (scan_all || !unique);
                 int bj = j1 < s.K ? j1 : 0;
@@ -661,12 +659,11 @@ encode_tensor_kernel(const Params p)
                     const float lim_s = __shfl_sync(0xFFFFFFFFu, lim, src);
                     const int cnt_s = __shfl_sync(0xFFFFFFFFu, cnt, src);
                     const uint32_t qmask_s = __shfl_sync(0xFFFFFFFFu, qmask, src);
-                    const uint32_t kmask_s = __shfl_sync(0xFFFFFFFFu, kmask, src);
+                    const uint32_t hmask_s = __shfl_sync(0xFFFFFFFFu, hmask, src);
                     const uint32_t bmask_s = __shfl_sync(0xFFFFFFFFu, bmask, src);
                     const bool all_s = __shfl_sync(0xFFFFFFFFu, (int)scan_all, src) != 0;
                     const int row_s = rloc - lane + src;
-                    const int lq = lane >= 30 ? 10 : lane / 3;
-                    const bool mine = ((qmask_s >> lq) & 1u) && ((kmask_s >> (lane - 3 * lq)) & 1u);
+                    const bool mine = ((qmask_s >> (lane & 15)) & 1u) && ((hmask_s >> (lane >> 4)) & 1u);
                     float bv = INFINITY;
                     int bi = 0x7FFFFFFF;
                     if (all_s) {

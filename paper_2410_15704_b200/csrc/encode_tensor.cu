@@ -376,8 +376,10 @@ encode_tensor_kernel(const Params p)
         // One thread per tile, each in a warp of its own so that the tiles' waits overlap.
         // Whatever it does between two tcgen05.mma chains delays its tile, so descriptors
         // are built once and all counters advance by increments.
-        if (lane == 0 && my_passes > 0) {
-            const int t = warp - kEpiThreads / 32;
+        // (The whole warp runs the loop with warp-uniform values and one lane issues: operands that the
+        // compiler knows to be uniform can stay in uniform registers, which tcgen05.mma reads directly.)
+        if (my_passes > 0) {
+            const int t = __shfl_sync(0xFFFFFFFFu, warp, 0) - kEpiThreads / 32;
             const uint32_t total = (uint32_t)my_passes * (uint32_t)s.R * (uint32_t)S;
             const uint32_t idesc = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);   // f16 x f16 -> f32, M=N=128
             // Seven K=16 steps: hi.hi (2), hi.lo (2), lo.hi (2) with A in TMEM (8 columns per
@@ -393,15 +395,17 @@ encode_tensor_kernel(const Params p)
             bool ok = true, first = true, active = t < work.round_size(0);
             for (uint32_t q = 0; q < total && ok; ++q) {
                 ok = mbar_wait(BAR(kBarFull + slot), full_par, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!active) {
                     // this tile sits the round out, but the slot still waits for its release
-                    if (ok) mbar_arrive(BAR(kBarEmpty + slot));
+                    if (ok && lane == 0) mbar_arrive(BAR(kBarEmpty + slot));
                     if (++slot == (uint32_t)kRing) { slot = 0; full_par ^= 1u; }
                     if (++in_round == per_round) { in_round = 0; ++round; active = round < work.rounds && t < work.round_size(round); }
                     continue;
                 }
                 if (ok && s_in == 0) ok = mbar_wait(bar_ready, ready_par, abort_flag);
                 if (ok && !first) ok = mbar_wait(bar_free, free_par, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 first = false;
                 tc_fence_after();
@@ -409,15 +413,18 @@ encode_tensor_kernel(const Params p)
                 // (self-test of the give-up path: the chain that nothing comes after is left out, so that the
                 // epilogue's wait for it runs out with no copy or MMA of this CTA still in flight)
                 if (p.drop_last_chain && t == 0 && q == total - 1) break;
-                mma_f16_ts(acc, a0, bd, idesc, 0);                      // hi[0:16]  . hi cells 0-1
-                mma_f16_ts(acc, a0 + 8, bd + 2 * 128, idesc, 1);        // hi[16:32] . hi cells 2-3
-                mma_f16_ts(acc, a0, bd + 4 * 128, idesc, 1);            // hi[0:16]  . lo cells 4-5
-                mma_f16_ts(acc, a0 + 8, bd + 6 * 128, idesc, 1);        // hi[16:32] . lo cells 6-7
-                mma_f16_ts(acc, a0 + 16, bd, idesc, 1);                 // lo[0:16]  . hi cells 0-1
-                mma_f16_ts(acc, a0 + 24, bd + 2 * 128, idesc, 1);       // lo[16:32] . hi cells 2-3
-                mma_f16_ss(acc, ones_desc, bd + 8 * 128, idesc, 1);     // (1 1 1 0..) . norm cells 8-9
-                mma_commit(bar_acc);
-                mma_commit(BAR(kBarEmpty + slot));
+                if (lane == 0) {
+                    mma_f16_ts(acc, a0, bd, idesc, 0);                      // hi[0:16]  . hi cells 0-1
+                    mma_f16_ts(acc, a0 + 8, bd + 2 * 128, idesc, 1);        // hi[16:32] . hi cells 2-3
+                    mma_f16_ts(acc, a0, bd + 4 * 128, idesc, 1);            // hi[0:16]  . lo cells 4-5
+                    mma_f16_ts(acc, a0 + 8, bd + 6 * 128, idesc, 1);        // hi[16:32] . lo cells 6-7
+                    mma_f16_ts(acc, a0 + 16, bd, idesc, 1);                 // lo[0:16]  . hi cells 0-1
+                    mma_f16_ts(acc, a0 + 24, bd + 2 * 128, idesc, 1);       // lo[16:32] . hi cells 2-3
+                    mma_f16_ss(acc, ones_desc, bd + 8 * 128, idesc, 1);     // (1 1 1 0..) . norm cells 8-9
+                    mma_commit(bar_acc);
+                    mma_commit(BAR(kBarEmpty + slot));
+                }
+                __syncwarp();
                 free_par ^= 1u;
                 if (++slot == (uint32_t)kRing) { slot = 0; full_par ^= 1u; }
                 if (++s_in == (uint32_t)S) { s_in = 0; ready_par ^= 1u; }

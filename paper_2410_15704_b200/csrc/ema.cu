@@ -178,12 +178,22 @@ ema_stats_quad_kernel(Shape s, const void *__restrict__ x, int64_t n, int64_t st
         const int my_bin = lane < per ? (lane % R) * s.K + (int)code : -1 - lane;   // (idle lanes: bins of their own)
         const uint32_t same = __match_any_sync(0xFFFFFFFFu, my_bin);
         if (lane < per && lane == __ffs(same) - 1) atomicAdd(&hist[my_bin], (uint32_t)__popc(same));
-        for (int r = 0; r < R; ++r) {
-            const uint32_t j = __shfl_sync(0xFFFFFFFFu, code, g * R + r);
-            const size_t at = ((size_t)r * s.K + j) * 32 + 4 * q;
-            const float4 e = __ldg(reinterpret_cast<const float4 *>(cb + at));
-            atomicAdd(reinterpret_cast<float4 *>(sum + at), make_float4(z[0], z[1], z[2], z[3]));
-            z[0] -= e.x; z[1] -= e.y; z[2] -= e.z; z[3] -= e.w;
+        // the codewords of all stages are asked for first (they depend on the codes only), then the
+        // residual walks through the stages (R <= 8 here: four groups, at most 32 codes)
+        size_t at[8];
+        float4 e[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const uint32_t j = __shfl_sync(0xFFFFFFFFu, code, g * R + (r < R ? r : 0));
+            at[r] = ((size_t)(r < R ? r : 0) * s.K + j) * 32 + 4 * q;
+            e[r] = __ldg(reinterpret_cast<const float4 *>(cb + at[r]));
+        }
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if (r < R) {
+                atomicAdd(reinterpret_cast<float4 *>(sum + at[r]), make_float4(z[0], z[1], z[2], z[3]));
+                z[0] -= e[r].x; z[1] -= e[r].y; z[2] -= e[r].z; z[3] -= e[r].w;
+            }
         }
     }
     __syncthreads();

@@ -44,10 +44,15 @@ def workload_name(tokens):
     return f"ema_learning batch: {tokens} tokens x 8 heads x 128 bf16, strided groups of 32, R=8, K=1024"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, per head vector,
-# from ncu captures of the kernels as they stand (zero entries: not captured since the kernel last changed).
-DRAM_TRAFFIC_PER_VECTOR = {
-    # kernel: (bytes per head vector, vectors of the captured launch)
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernels, from ncu captures of the
+# kernels as they stand, keyed by (kernel, workload, tokens): an entry holds for that launch only, any other size
+# reports null.  An entry is taken out when its kernel changes.
+DRAM_TRAFFIC = {
+    # encode with the EMA statistics fused in: 273.0 MB read + 55.5 MB written over 1,048,576 head vectors
+    ("encode_tensor_kernel", "ema_learning", 131072): 273005312 + 55478016,
+    # decode, strided layout: 70.0 MB read + 214.3 MB written (the rest of the 268 MB output still sat in L2
+    # when the kernel ended)
+    ("decode_quoted_kernel", "decode_bandwidth", 131072): 70017280 + 214340608,
 }
 
 
@@ -440,7 +445,7 @@ def run_ours(args):
     enc_tflops = alg["encode_flops"] / (enc_ms * 1e-3) / 1e12
     # the encode kernel runs for milliseconds at a time, back to back for seconds: the sustained peak applies
     tensor_peak = peaks["bf16_tflops_sustained"]
-    traffic = DRAM_TRAFFIC_PER_VECTOR.get("encode_tensor_kernel")
+    traffic = DRAM_TRAFFIC.get(("encode_tensor_kernel", "ema_learning", args.tokens))
     line = {
         "metric": METRIC, "value": n * world * args.steps / (total_ms * 1e-3) / 1e6, "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -463,10 +468,9 @@ def run_ours(args):
         "roofline": {"kernel": "encode_tensor_kernel", "bound": "tensor", "achieved": enc_tflops, "peak": tensor_peak,
                      "unit": "TFLOP/s", "frac": enc_tflops / tensor_peak,
                      "frac_of_burst_peak": enc_tflops / peaks["bf16_tflops"],
-                     "traffic": None if traffic is None else int(traffic[0] * n),
-                     "traffic_note": ("no ncu capture of this kernel as it stands" if traffic is None else
-                                      f"{traffic[0]:.1f} B per head vector from a capture of {traffic[1]} vectors, "
-                                      "scaled by the vectors of this launch"),
+                     "traffic": traffic,
+                     "traffic_note": ("no ncu capture of this kernel at this size" if traffic is None else
+                                      "dram bytes read + written by one launch of this size under ncu"),
                      "peak_source": f"{peaks['source']} bf16 sustained x1 (f16 operands, same rate)"},
         "e2e": {"value": n * world * args.steps / (e2e_ms * 1e-3) / 1e6, "unit": UNIT,
                 "h2d_bytes_per_step": x_host.numel() * 2,
@@ -485,11 +489,12 @@ def run_ours(args):
         side = side_workloads(torch, rvq, peaks, flush)
         line["configs"] = side
         d4 = side["decode_bandwidth"][side["decode_bandwidth"]["headline"]]
-        dtraffic = DRAM_TRAFFIC_PER_VECTOR.get("decode_sliced_kernel")
-        line["roofline_decode"] = {"kernel": "decode_sliced_kernel", "workload": "decode_bandwidth, " + side["decode_bandwidth"]["headline"],
+        dtraffic = DRAM_TRAFFIC.get(("decode_quoted_kernel", "decode_bandwidth", 131072))
+        line["roofline_decode"] = {"kernel": "decode_quoted_kernel", "workload": "decode_bandwidth, " + side["decode_bandwidth"]["headline"],
                                    "bound": "hbm", "achieved": d4["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                    "frac": d4["frac_hbm"],
-                                   "traffic": None if dtraffic is None else int(dtraffic[0] * 1048576),
+                                   "traffic": dtraffic,
+                                   "traffic_note": "dram bytes read + written by one launch under ncu, strided layout",
                                    "peak_source": f"{peaks['source']} copy bandwidth"}
 
     if world == 1 and not args.no_cpu_baseline:

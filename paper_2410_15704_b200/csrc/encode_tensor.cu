@@ -2,8 +2,10 @@
 //
 // One persistent CTA per SM takes a contiguous run of 128-row tiles and works
 // through it in rounds of up to three tiles (one row per thread, 12 epilogue
-// warps; rounds are sized evenly, e.g. 7 tiles = 3 + 2 + 2) plus four single-thread roles in
-// warps of their own: one MMA issuer per tile and the operand loader.
+// warps; rounds are sized evenly, e.g. 7 tiles = 3 + 2 + 2) plus four role
+// warps: one MMA issuer per tile (the warp runs its loop as one, a single lane
+// issues) and the operand loader.  The role warps give registers up
+// (setmaxnreg 40) and the epilogue warps take them (152).
 //   - Scores ||e||^2 - 2 z.e of a 128-row tile against 128 codewords are one
 //     tcgen05.mma chain (M=128, N=128, seven K=16 steps over the split
 //     half-precision operands described in prepare.cu), accumulated in float32
@@ -11,14 +13,20 @@
 //   - The B operand (128 codewords per slot) streams from the prepared block
 //     through a ring of shared-memory slots filled by cp.async.bulk; every
 //     slot serves all three tiles.
-//   - Epilogue threads read their row's 128 scores with tcgen05.ld (the next
-//     32 columns are in flight while the current 32 are reduced) and keep
-//     (i) the minimum of every 32-column block that comes within the error
-//     window of the running minimum, and (ii) the minimum per 3-column cell
-//     position over all blocks.  Any column that could be the exact argmin lies
-//     in a listed block at a listed cell position; those few columns are
-//     re-scored exactly in float32 against the float32 codebook (direct form,
-//     lowest index on ties), so the emitted code is the exact-L2 choice.
+//   - Epilogue threads read their row's 128 scores with four tcgen05.ld of 32
+//     columns issued together, hand the accumulator back to the issuer as soon
+//     as they have landed, and fold them afterwards while the next chain runs.
+//     The fold keeps running minima over four partitions of the stage's
+//     columns: by 128-column chunk (a short list of the chunks that come within
+//     the error window of the running minimum), by 32-column block of a chunk,
+//     by half of a block, and by place within a half (16 places): 36 minimum
+//     operations per 32 scores.  At the stage end the sets of chunks, blocks,
+//     halves and places whose minimum lies inside the window bound where the
+//     exact argmin can be: when each set has one member the column is known
+//     and only that codeword is fetched; otherwise the warp re-scores every
+//     column in the product of the sets exactly in float32 against the float32
+//     codebook (direct form, lowest index on ties), and a full exact scan
+//     covers list overflow.  The emitted code is the exact-L2 choice.
 //   - The A operand (the residual split into half-precision head and remainder)
 //     lives in TMEM next to its tile's scores, so the tensor core fetches only B
 //     from shared memory; the constant (1 1 1 0 ...) rows that pick up the
@@ -296,7 +304,8 @@ struct Work {
     __device__ __forceinline__ int round_first(int k) const { return first + k * (count / rounds) + min(k, count % rounds); }
 };
 
-// 17 warps are granted registers as 20 (whole groups of four): 96 per thread.
+// 16 warps, launched with 128 registers per thread; the four role warps then keep 40 each and the
+// twelve epilogue warps take 152 (4 x 40 + 12 x 152 = 1984 of the 2048 per lane).
 __global__ void __launch_bounds__(kThreads, 1)
 encode_tensor_kernel(const Params p)
 {

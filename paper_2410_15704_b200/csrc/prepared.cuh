@@ -58,8 +58,9 @@ constexpr int kDecodeExactK = 3584;                       // ... 64 bytes per co
 //     (4 channels per slice up to kDecodeExactWideK, 2 beyond);
 //   - 16-bit level tables (16-bit outputs only: their own rounding, 2^-9 or 2^-12 relative, dwarfs the
 //     tables') fit up to kDecodeMaxK codes and are the faster ones while the deviations are moderate;
-//   - where both fit (16-bit outputs, up to kDecodeMaxK codes) both kernels are launched and the one the
-//     deviations do not call for returns at once.
+//   - where both fit (16-bit outputs, up to kDecodeMaxK codes) a sample of the deviations decides on the
+//     device: four groups at depth 8 in one launch that holds all three kinds of table, other shapes as
+//     two launches of which the one not called for returns at once.
 __host__ __device__ inline bool decode_exact_tables(const Shape &s)
 {
     return s.gd == 32 && s.G <= 32 && (s.G & (s.G - 1)) == 0 && s.R <= 8 && s.K <= kDecodeExactK;

@@ -178,10 +178,15 @@ int rvq_encode_exact(const rvq_config *cfg /* host */, const void *x, int64_t n,
  * copies (up to 3584 codes per stage) or, for 16-bit outputs and up to 3072
  * codes, 16-bit levels of each stage's value range kept in the prepared block.
  * With the levels the sum before the multiplication by std is within
- * err <= 1.04 * sum_r (max C_r - min C_r) * 2^-17 of the float32 one; a head vector whose
- * std would make std * err exceed 0.9e-3 gets the float32 sum instead, so the
- * value before the final rounding is always within 1e-3 of the exact one.  Other
- * shapes gather the float32 codebooks from global memory.
+ * err <= 1.04 * sum_r (max C_r - min C_r) * 2^-17 of the float32 one (levels of
+ * each stage's own range), or within 4.1 * sum_r (max C_r - min C_r) * 2^-17 (levels
+ * on a unit shared by the stages of one parity, which a decoder adds as packed
+ * integers; four groups at depth 8).  The call looks at a sample of the deviations
+ * and takes the coarsest table that keeps std * err below 0.9e-3, or the float32
+ * tables; a single head vector whose std would still make std * err exceed 0.9e-3
+ * gets the float32 sum instead, so the value before the final rounding is always
+ * within 1e-3 of the exact one.  Other shapes gather the float32 codebooks from
+ * global memory.
  *   codes, std_f16  in   as produced by rvq_encode
  *   x_out           out  n rows of x_dtype, row v at element v * out_row_stride
  * A code >= K is read as code 0 and counted in status->bad_codes.

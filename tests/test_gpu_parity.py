@@ -356,6 +356,32 @@ def test_tensor_encode_at_the_edge_of_its_error_window():
           f"re-scored {st['rescored_rows']}")
 
 
+@pytest.mark.parametrize("K", [100, 300])
+def test_padding_columns_never_decide_a_code(K):
+    """A codebook size that is no multiple of 128 leaves padded columns in the last operand slot,
+    scored with a large constant.  Rows that are far from every codeword (all codewords in one
+    orthant, the scaled rows large and pointing the other way) score above that constant on every
+    real column; the code must still be the exact argmin (Algorithm 1), as the all-float32 kernel
+    and the oracle choose it."""
+    g = np.random.default_rng(K)
+    cb = g.uniform(0.8, 1.5, size=(2, K, 32)).astype(np.float32)
+    cb[1] *= 0.1 * g.choice([-1.0, 1.0], size=(K, 32)).astype(np.float32)
+    n = 2048
+    x = -(1.0 + 6e-4 * g.normal(size=(n, 128))).astype(np.float32)       # scaled rows of about -1500 per channel
+    x[::7] = g.normal(size=(len(x[::7]), 128)).astype(np.float32)        # ordinary rows in between
+    cfg = rvq.make_config(128, 32, rvq.CONTIGUOUS, 2, K, 16, rvq.F32, 0)
+    xd = torch.from_numpy(x).cuda()
+    codes, std_bits, st, b = gpu_encode(cfg, xd, n, cb)
+    exact = torch.empty_like(b.codes)
+    rvq.rvq_encode_exact(cfg, xd, n, 128, b.codebooks, b.prepared, exact, b.std, b.status)
+    torch.cuda.synchronize()
+    assert torch.equal(b.codes, exact)
+    assert_codes_match(x, codes, cb, rvq.CONTIGUOUS)
+    z = oracle.scaled_groups(x[1:2], 32, rvq.CONTIGUOUS)
+    assert np.min(((z[:, None, :] - cb[0][None].astype(np.float64)) ** 2).sum(-1) - (z ** 2).sum(-1)[:, None]) > 60000.0
+    assert st["wait_timeouts"] == 0
+
+
 @pytest.mark.parametrize("which", ["tensor", "exact", "stats"])
 def test_stage_energy_matches_oracle_prefixes(which):
     """stage_energy[r] is the squared norm of what stage r leaves, summed over the batch: the

@@ -211,11 +211,12 @@ int rvq_decode(const rvq_config *cfg /* host */, const void *codes, const uint16
  *                             rvq_rope_table
  *   prepared              in  block of rvq_prepare_codebooks for these codebooks, or NULL
  * Two or more groups of 32 (a power-of-two number) with depth <= 8: up to 3584 codes per stage float32
- * shared-memory tables (exact float32 sums); with 16-bit outputs, a prepared block and
- * 1537..3072 codes also the level tables described under rvq_decode, chosen when the
- * deviations are moderate (a head vector whose std would make std * err exceed 0.6e-3
- * gets float32 sums, so the rotated value before the final rounding stays within 1e-3
- * of the exact one).  Other shapes gather from global memory.
+ * shared-memory tables (exact float32 sums); with 16-bit outputs and a prepared block also
+ * the level tables described under rvq_decode (dim 128 at depth 8 with up to 1536 codes:
+ * both kinds of level table, 8-channel slices, one launch; 1537..3072 codes: the per-stage
+ * levels), chosen when the deviations are moderate (a head vector whose std would make
+ * std * err exceed 0.6e-3 gets float32 sums, so the rotated value before the final
+ * rounding stays within 1e-3 of the exact one).  Other shapes gather from global memory.
  */
 enum { RVQ_ROPE_HALVES = 0, RVQ_ROPE_ADJACENT = 1 };
 int rvq_decode_rope(const rvq_config *cfg /* host */, const void *codes, const uint16_t *std_f16,

@@ -486,12 +486,36 @@ decode_sliced_body(const Shape &s, const void *__restrict__ codes, const uint16_
 // SUMMED: the tables whose levels add up within 16 bits per stage parity (prepared.cuh): the table
 // words of the even steps and of the odd steps are added as they are (which parity of stages a
 // thread's even steps are depends on its lane), and scaled once per parity.
-template <int DT, int CH, int LAYOUT, int BITS, bool SUMMED>
+// ROPE (8-channel slices): the rotary embedding is applied to the float32 results before the one
+// rounding (1: pairs are channels (k, k + 64), 2: (2k, 2k + 1)).  The partner of a channel is in the
+// same thread (adjacent pairs on contiguous groups), in the lane of another group of the same head
+// vector (half-split pairs on contiguous groups: lane g ^ 2; adjacent pairs on strided groups: lane
+// g ^ 1), or -- half-split pairs on strided groups, where the partner of element i of a group is
+// element i + 16 of the same group -- brought into the thread by making a slice the elements
+// {4 sl .. 4 sl + 3} and {4 sl + 16 .. 4 sl + 19} instead of eight consecutive ones.
+// Lanes g = 0..3 of a head vector hold the elements (e0, e1) and (e2, e3) of their group as two packed
+// words; lane L gets back element L of the groups 0..3 (four consecutive channels of a strided row).
+__device__ __forceinline__ uint2 transpose_group_elements(uint32_t w0, uint32_t w1, uint32_t g)
+{
+    const bool b1 = g & 1u, b2 = g & 2u;
+    const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, b2 ? w0 : w1, 2);
+    // lanes 0, 1 now hold (e0, e1) of groups g and g + 2; lanes 2, 3 hold (e2, e3) of g - 2 and g
+    const uint32_t lo_g = b2 ? r0 : w0, hi_g = b2 ? w1 : r0;
+    const uint32_t keep = __byte_perm(lo_g, hi_g, b1 ? 0x7632 : 0x5410);
+    const uint32_t send = __byte_perm(lo_g, hi_g, b1 ? 0x5410 : 0x7632);
+    const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+    const uint32_t even = b1 ? got : keep, odd = b1 ? keep : got;       // groups (0, 2) and (1, 3)
+    return make_uint2(__byte_perm(even, odd, 0x5410), __byte_perm(even, odd, 0x7632));
+}
+
+template <int DT, int CH, int LAYOUT, int BITS, bool SUMMED, int ROPE = 0>
 __device__ __forceinline__ void
 decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
                    const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
-                   int64_t stride, rvq_status *st, uint8_t *table)
+                   int64_t stride, rvq_status *st, uint8_t *table, RopeArgs ra = RopeArgs())
 {
+    static_assert(ROPE == 0 || CH == 8, "the rotary variant uses 8-channel slices");
+    constexpr bool SPLIT = ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED;   // slice = two runs of four elements
     constexpr int NS = 32 / CH;                                  // slices
     if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;
     constexpr uint32_t kEntry = 2 * CH, kLine = 8 * kEntry;      // bytes per (code, stage) and per code: 128 or 64
@@ -503,7 +527,20 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
         const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256 + (SUMMED ? decode_table_bytes(s.K) : 0)) +
                            (size_t)slice * s.K * CH;
         uint4 *dst = reinterpret_cast<uint4 *>(table);
-        for (uint32_t t = tid; t < (uint32_t)s.K * CH; t += kDecThreads) dst[t] = __ldg(src + t);
+        if (SPLIT) {
+            // entry (code, stage) = elements 4 slice .. + 3 (half of the entry of slice / 2 in the prepared
+            // table) followed by their partners 16 elements on (the same half of the entry of slice / 2 + 2)
+            const uint2 *half = reinterpret_cast<const uint2 *>(dsec + 256 + (SUMMED ? decode_table_bytes(s.K) : 0));
+            const size_t per_slice = (size_t)s.K * 8;            // entries of one slice
+            const uint2 *sa = half + ((size_t)(slice >> 1) * per_slice) * 2 + (slice & 1u);
+            const uint2 *sb = half + ((size_t)((slice >> 1) + 2) * per_slice) * 2 + (slice & 1u);
+            for (uint32_t t = tid; t < (uint32_t)s.K * 8; t += kDecThreads) {
+                const uint2 a = __ldg(sa + 2 * (size_t)t), b = __ldg(sb + 2 * (size_t)t);
+                dst[t] = make_uint4(a.x, a.y, b.x, b.y);
+            }
+        } else {
+            for (uint32_t t = tid; t < (uint32_t)s.K * CH; t += kDecThreads) dst[t] = __ldg(src + t);
+        }
     }
     // this thread visits stage (rot + k) & 7 at step k (the 8 lanes of a quarter warp then touch 8
     // different bank groups): the scale of that stage in bytes 0 and 3, and the byte offset of its entry
@@ -518,7 +555,7 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
     }
     const float bias = dp->bias, base = SUMMED ? dp->pbase : dp->base;
     const float terr = SUMMED ? dp->perr : dp->err;
-    const float exact_above = terr > 0.0f ? 0.9e-3f / terr : INFINITY;
+    const float exact_above = terr > 0.0f ? (ROPE != 0 ? 0.6e-3f : 0.9e-3f) / terr : INFINITY;   // (a rotation adds two table errors)
     const uint32_t Ku = (uint32_t)s.K;
     __syncthreads();
 
@@ -527,12 +564,14 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
     uint32_t bad = 0;
     // The codes and the deviation of a row are fetched one iteration ahead, so that their latency is
     // spent while the previous row's table entries are gathered.
-    auto fetch = [&](uint32_t row, uint32_t &c0, uint32_t &c1, uint32_t &c2, uint32_t &c3, uint16_t &sdb) {
+    auto fetch = [&](uint32_t row, uint32_t &c0, uint32_t &c1, uint32_t &c2, uint32_t &c3, uint16_t &sdb, int &posv) {
         c0 = c1 = c2 = c3 = 0u;
         sdb = 0;
+        posv = 0;
         if (row >= rows) return;
         const uint32_t v = row >> 2, g = row & 3u;
         sdb = __ldg(std16 + v);
+        if (ROPE != 0) posv = __ldg(ra.position + (ra.shift >= 0 ? v >> ra.shift : v / (uint32_t)ra.per_position));
         if (BITS == 16) {
             const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + row);
             c0 = c.x; c1 = c.y; c2 = c.z; c3 = c.w;
@@ -549,7 +588,8 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
     };
     uint32_t p0, p1, p2, p3;
     uint16_t psd;
-    fetch(part * kDecThreads + tid, p0, p1, p2, p3, psd);
+    int ppos;
+    fetch(part * kDecThreads + tid, p0, p1, p2, p3, psd, ppos);
     for (uint32_t row = part * kDecThreads + tid; row - tid < rows; row += parts * kDecThreads) {
         // (the loop bound keeps whole warps together for the shuffles below)
         const bool live = row < rows;
@@ -557,7 +597,17 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
         // the 8 codes of this row as 4 words, stage r in half r
         uint32_t c0 = p0, c1 = p1, c2 = p2, c3 = p3;
         const uint16_t sdb = psd;
-        fetch(row + parts * kDecThreads, p0, p1, p2, p3, psd);
+        // rotary decode: the row of (cos, sin) pairs of this head vector's position; the 128-byte line
+        // that holds this thread's pairs is asked into L1 now and read after the gather
+        const float2 *cs = nullptr;
+        if (ROPE != 0) {
+            cs = ra.table + (size_t)min(max(ppos, 0), ra.positions - 1) * 64;
+            const float2 *mine = ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED ? cs + 16 * slice
+                                 : ROPE == 2 && LAYOUT == RVQ_GROUP_CONTIGUOUS ? cs + g * 16 + slice * 4
+                                 : ROPE == 1 ? cs + (g & 1u) * 32 + slice * 8 : cs + 16 * slice;
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(mine));
+        }
+        fetch(row + parts * kDecThreads, p0, p1, p2, p3, psd, ppos);
         if (BITS != 16) {
             // shift the window down to bit 0 and cut the codes out of it at offsets known at compile time
             const uint32_t sh = (g * (8u * BITS)) & 31u;
@@ -645,21 +695,75 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
             for (int r = 0; r < 8; ++r) {
                 uint32_t j = (r & 1) ? (cn[r >> 1] >> 16) : (cn[r >> 1] & 0xFFFFu);
                 if (j >= Ku) j = 0;
-                const float4 *e = reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * 32 + slice * CH);
+                const float4 *e = reinterpret_cast<const float4 *>(cb + ((size_t)r * s.K + j) * 32 + (SPLIT ? slice * 4 : slice * CH));
 #pragma unroll
                 for (int q = 0; q < CH / 4; ++q) {
-                    const float4 t = __ldg(e + q);
+                    const float4 t = __ldg(e + (SPLIT ? 4 * q : q));
                     ex[4 * q] += t.x; ex[4 * q + 1] += t.y; ex[4 * q + 2] += t.z; ex[4 * q + 3] += t.w;
                 }
             }
 #pragma unroll
             for (int i = 0; i < CH; ++i) o8[i] = ex[i] * sd;
         }
+        if (ROPE != 0) {
+            // (cos, sin) of the pairs of this thread's channels
+            if (ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED) {
+                // places 0..3 are channels 4 (4 slice + i) + g = pair index; places 4..7 their partners 64 on
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 c = __ldg(cs + (4 * slice + i) * 4 + g);
+                    const float a = o8[i], b = o8[i + 4];
+                    o8[i] = a * c.x - b * c.y;
+                    o8[i + 4] = b * c.x + a * c.y;
+                }
+            } else if (ROPE == 2 && LAYOUT == RVQ_GROUP_CONTIGUOUS) {
+                // channels 32 g + 8 slice + i: pairs 16 g + 4 slice + i / 2, both halves in this thread
+                const float4 *q = reinterpret_cast<const float4 *>(cs + g * 16 + slice * 4);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float4 c = __ldg(q + h);
+                    const float a0 = o8[4 * h], b0 = o8[4 * h + 1], a1 = o8[4 * h + 2], b1 = o8[4 * h + 3];
+                    o8[4 * h] = a0 * c.x - b0 * c.y;     o8[4 * h + 1] = b0 * c.x + a0 * c.y;
+                    o8[4 * h + 2] = a1 * c.z - b1 * c.w; o8[4 * h + 3] = b1 * c.z + a1 * c.w;
+                }
+            } else if (ROPE == 1) {
+                // contiguous groups, pairs (k, k + 64): the partner is the same place of group g ^ 2;
+                // pairs 32 (g & 1) + 8 slice + i
+                const float4 *q = reinterpret_cast<const float4 *>(cs + (g & 1u) * 32 + slice * 8);
+                const bool first = (g & 2u) == 0;
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const float4 c = __ldg(q + h);
+                    const float p0 = __shfl_xor_sync(0xFFFFFFFFu, o8[2 * h], 2);
+                    const float p1 = __shfl_xor_sync(0xFFFFFFFFu, o8[2 * h + 1], 2);
+                    o8[2 * h] = first ? o8[2 * h] * c.x - p0 * c.y : o8[2 * h] * c.x + p0 * c.y;
+                    o8[2 * h + 1] = first ? o8[2 * h + 1] * c.z - p1 * c.w : o8[2 * h + 1] * c.z + p1 * c.w;
+                }
+            } else {
+                // strided groups, pairs (2k, 2k + 1): channels 4 e + g and 4 e + (g ^ 1), e = 8 slice + i;
+                // pair 2 e + g / 2
+                const bool first = (g & 1u) == 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float2 c = __ldg(cs + 2 * (8 * slice + i) + (g >> 1));
+                    const float p = __shfl_xor_sync(0xFFFFFFFFu, o8[i], 1);
+                    o8[i] = first ? o8[i] * c.x - p * c.y : o8[i] * c.x + p * c.y;
+                }
+            }
+        }
         uint32_t w[CH / 2];
 #pragma unroll
         for (int c = 0; c < CH / 2; ++c) w[c] = Out<DT>::pack(o8[2 * c], o8[2 * c + 1]);
         uint16_t *o16 = reinterpret_cast<uint16_t *>(out) + (size_t)v * stride;
-        if (LAYOUT == RVQ_GROUP_CONTIGUOUS) {
+        if (SPLIT) {
+            // lane L stores element 4 slice + L of the four groups, and its partner 16 elements on
+            const uint2 lo = transpose_group_elements(w[0], w[1], g);
+            const uint2 hi = transpose_group_elements(w[CH / 2 - 2], w[CH / 2 - 1], g);
+            if (live) {
+                *reinterpret_cast<uint2 *>(o16 + 4 * (4 * slice + g)) = lo;
+                *reinterpret_cast<uint2 *>(o16 + 4 * (16 + 4 * slice + g)) = hi;
+            }
+        } else if (LAYOUT == RVQ_GROUP_CONTIGUOUS) {
             if (live) {
                 if (CH == 8)
                     *reinterpret_cast<uint4 *>(o16 + g * 32 + slice * 8) = make_uint4(w[0], w[1], w[CH / 2 - 2], w[CH / 2 - 1]);
@@ -732,18 +836,21 @@ decode_sliced_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
 }
 
 // 0: summed-level tables, 1: per-stage scaled levels, 2: float32 tables -- the first kind within whose reach
-// at least seven eighths of a sample of up to 256 deviations lie.  Uniform over all CTAs of a launch.
-__device__ __forceinline__ int sample_table_kind(const uint16_t *__restrict__ std16, int64_t n, const uint8_t *__restrict__ dsec)
+// all but one in 64 of a sample of up to 256 deviations lie.  Uniform over all CTAs of a launch.
+__device__ __forceinline__ int sample_table_kind(const uint16_t *__restrict__ std16, int64_t n, const uint8_t *__restrict__ dsec,
+                                                 float reach = 0.9e-3f)
 {
     const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
-    const float above_l = dp->err > 0.0f ? 0.9e-3f / dp->err : INFINITY;
-    const float above_s = dp->perr > 0.0f ? 0.9e-3f / dp->perr : INFINITY;
+    const float above_l = dp->err > 0.0f ? reach / dp->err : INFINITY;
+    const float above_s = dp->perr > 0.0f ? reach / dp->perr : INFINITY;
     const int64_t samples = n < 256 ? n : 256, every = n < 256 ? 1 : n >> 8;
     const float sd = threadIdx.x < samples ? fabsf(__half2float(__ushort_as_half(std16[threadIdx.x * every]))) : 0.0f;
     const int far_s = __syncthreads_count(sd > above_s);
     const int far_l = __syncthreads_count(sd > above_l);
-    if ((int64_t)far_s * 8 <= samples) return 0;
-    return (int64_t)far_l * 8 <= samples ? 1 : 2;
+    // (a row beyond a table's reach takes the exact route, and its whole warp of eight head vectors waits
+    // for it: a table is taken only while at most one sampled row in 64 is beyond it)
+    if ((int64_t)far_s * 64 <= samples) return 0;
+    return (int64_t)far_l * 64 <= samples ? 1 : 2;
 }
 
 // One launch for the quoted shapes (dim 128, depth 8, 16-bit outputs, up to 3072 codes): every CTA
@@ -763,6 +870,25 @@ decode_quoted_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
         decode_levels_fast<DT, LCH, LAYOUT, BITS, false>(s, codes, std16, n, dsec, cb, out, stride, st, table);
     else
         decode_levels_fast<DT, LCH, LAYOUT, BITS, true>(s, codes, std16, n, dsec, cb, out, stride, st, table);
+}
+
+// The rotary decode of the quoted shapes (dim 128, depth 8, 16-bit outputs, up to 1536 codes, a prepared
+// block): one launch that takes the level tables with 8-channel slices while the deviations allow it (a
+// rotation adds two table errors, so their reach is 0.6e-3) and the float32 tables otherwise.
+template <int DT, int LAYOUT, int BITS, int ROPE>
+__global__ void __launch_bounds__(kDecThreads, 1)
+decode_rope_quoted_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
+                          const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
+                          int64_t stride, rvq_status *st, RopeArgs ra)
+{
+    extern __shared__ __align__(128) uint8_t table[];
+    const int kind = sample_table_kind(std16, n, dsec, 0.6e-3f);
+    if (kind == 2)
+        decode_sliced_body<DT, 4, true, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
+    else if (kind == 1)
+        decode_levels_fast<DT, 8, LAYOUT, BITS, false, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
+    else
+        decode_levels_fast<DT, 8, LAYOUT, BITS, true, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
 }
 
 // Decode with the rotary embedding, 4-channel slices (dim 128): float32 tables up to 1792 codes per stage,
@@ -880,6 +1006,30 @@ int launch_decode_rope(const Shape &s, const void *codes, const uint16_t *std16,
     if (levels)
         dsec = reinterpret_cast<const uint8_t *>(prepared) + (kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256;
     const int64_t tiles = (n * s.G + kDecThreads - 1) / kDecThreads;
+    // the quoted shapes with a prepared block: one launch, tables chosen on the device
+    if (prepared != nullptr && decode_levels_supported(s) && s.dim == 128 && s.G == 4 && s.R == 8 && s.K <= kDecodeWideK &&
+        n * 4 < 0x7FFFFFFFLL && (s.bits == 16 || s.bits == 10 || s.bits == 11)) {
+        const uint8_t *d = reinterpret_cast<const uint8_t *>(prepared) +
+                           (kPreparedImageOffset + encode_image_bytes(s) + 255) / 256 * 256;
+        auto quoted = [&](auto kernel) -> int {
+            const size_t smem = (size_t)s.K * 128;               // 8 channels of levels or 4 of float32 per code
+            const int grid = sms < 8 ? 8 : sms;
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return RVQ_ERR_LAUNCH;
+            kernel<<<grid, kDecThreads, smem, stream>>>(s, codes, std16, n, d, cb, out, stride, st, ra);
+            return check_launch();
+        };
+#define RVQ_RQ3(DT, LAY, ROPE)                                                                                       \
+        (s.bits == 16 ? quoted(decode_rope_quoted_kernel<DT, LAY, 16, ROPE>)                                         \
+         : s.bits == 10 ? quoted(decode_rope_quoted_kernel<DT, LAY, 10, ROPE>)                                       \
+                        : quoted(decode_rope_quoted_kernel<DT, LAY, 11, ROPE>))
+#define RVQ_RQ2(DT, LAY) (style == 0 ? RVQ_RQ3(DT, LAY, 1) : RVQ_RQ3(DT, LAY, 2))
+#define RVQ_RQ1(DT) (s.layout == RVQ_GROUP_CONTIGUOUS ? RVQ_RQ2(DT, RVQ_GROUP_CONTIGUOUS) : RVQ_RQ2(DT, RVQ_GROUP_STRIDED))
+        return s.dtype == RVQ_BF16 ? RVQ_RQ1(RVQ_BF16) : RVQ_RQ1(RVQ_F16);
+#undef RVQ_RQ1
+#undef RVQ_RQ2
+#undef RVQ_RQ3
+    }
     auto launch = [&](auto kernel, int ch, bool f32_tables) -> int {
         const int ns = 32 / ch;
         const size_t smem = (size_t)s.K * (f32_tables ? 32 : 16) * ch;

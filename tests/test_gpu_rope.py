@@ -29,11 +29,14 @@ def test_rope_table_matches_double_precision():
 
 
 def run_case(dim, gd, R, K, bits, layout, dtype, pairing, tokens=333, heads=8, max_pos=100000, with_prepared=True,
-             std_scale=1.0):
+             std_scale=1.0, outlier_every=0):
     g = np.random.default_rng(dim + K + R + layout * 7 + pairing)
     n, G = tokens * heads, dim // gd
     codes = g.integers(0, K, size=(n, G, R)).astype(np.int32)
-    std_bits = (std_scale * (np.abs(1.0 + 0.25 * g.normal(size=n)) + 0.05)).astype(np.float16).view(np.uint16)
+    std = std_scale * (np.abs(1.0 + 0.25 * g.normal(size=n)) + 0.05)
+    if outlier_every:
+        std[::outlier_every] *= 50.0                                     # single rows beyond the chosen table's reach
+    std_bits = std.astype(np.float16).view(np.uint16)
     cb = np.stack([g.normal(scale=0.5 * 0.75 ** r, size=(K, gd)) for r in range(R)]).astype(np.float32)
     pos = g.integers(0, max_pos, size=tokens).astype(np.int32)
     pos[:3] = [0, max_pos - 1, 1]
@@ -95,6 +98,20 @@ def test_decode_rope_level_tables(layout, pairing):
     # float32 tables with 2-channel slices: float32 outputs, and 16-bit outputs without a prepared block
     run_case(128, 32, 8, 2048, 11, layout, "f32", pairing, tokens=57)
     run_case(128, 32, 8, 3584, 12, layout, "bf16", pairing, tokens=57, with_prepared=False)
+
+
+@pytest.mark.parametrize("layout", [rvq_synth.CONTIGUOUS, rvq_synth.STRIDED])
+@pytest.mark.parametrize("pairing", [rvq.ROPE_HALVES, rvq.ROPE_ADJACENT])
+def test_decode_rope_quoted_shapes_take_every_kind_of_table(layout, pairing):
+    """dim 128, depth 8, up to 1536 codes, 16-bit outputs and a prepared block: one launch that picks the
+    summed levels (small deviations), the per-stage levels (moderate), or the float32 tables (large); uint16
+    and packed codes; a mixed batch sends single rows down the exact route."""
+    for std_scale in (0.3, 1.0, 3.0, 40.0):
+        run_case(128, 32, 8, 1024, 16, layout, "bf16", pairing, tokens=333, std_scale=std_scale)
+    run_case(128, 32, 8, 1024, 10, layout, "f16", pairing, tokens=131, std_scale=0.3)
+    run_case(128, 32, 8, 1536, 11, layout, "bf16", pairing, tokens=131, std_scale=1.0)
+    run_case(128, 32, 8, 1000, 10, layout, "bf16", pairing, tokens=57, std_scale=2.0)
+    run_case(128, 32, 8, 1024, 16, layout, "f16", pairing, tokens=131, std_scale=1.0, outlier_every=11)
 
 
 def test_decode_rope_clamps_positions_and_rejects_bad_arguments():

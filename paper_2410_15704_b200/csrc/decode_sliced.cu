@@ -508,18 +508,22 @@ __device__ __forceinline__ uint2 transpose_group_elements(uint32_t w0, uint32_t 
     return make_uint2(__byte_perm(even, odd, 0x5410), __byte_perm(even, odd, 0x7632));
 }
 
-template <int DT, int CH, int LAYOUT, int BITS, bool SUMMED, int ROPE = 0>
+// F32 (4 channels per slice): the table holds the float32 codeword channels themselves (16 bytes per
+// code and stage, the geometry of the 8-channel level tables), filled from the codebooks by the CTA;
+// exact float32 sums, no table error and no exact route.
+template <int DT, int CH, int LAYOUT, int BITS, bool SUMMED, int ROPE = 0, bool F32 = false>
 __device__ __forceinline__ void
 decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_t *__restrict__ std16, int64_t n,
                    const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
                    int64_t stride, rvq_status *st, uint8_t *table, RopeArgs ra = RopeArgs())
 {
     static_assert(ROPE == 0 || CH == 8, "the rotary variant uses 8-channel slices");
+    static_assert(!F32 || (CH == 4 && !SUMMED && ROPE == 0), "float32 tables: 4-channel slices, no rotation here");
     constexpr bool SPLIT = ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED;   // slice = two runs of four elements
     constexpr int NS = 32 / CH;                                  // slices
     if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;
-    constexpr uint32_t kEntry = 2 * CH, kLine = 8 * kEntry;      // bytes per (code, stage) and per code: 128 or 64
-    constexpr int kShift = CH == 8 ? 7 : 6;                      // log2(kLine)
+    constexpr uint32_t kEntry = F32 ? 16 : 2 * CH;               // bytes per (code, stage); a code's line is 8 entries
+    constexpr int kShift = (F32 || CH == 8) ? 7 : 6;             // log2 of the line's bytes
     const DecodeParams *dp = reinterpret_cast<const DecodeParams *>(dsec);
     const uint32_t slice = blockIdx.x % NS, part = blockIdx.x / NS, parts = gridDim.x / NS;
     const uint32_t tid = threadIdx.x, lane = tid & 31u, rot = lane & 7u;
@@ -527,7 +531,13 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
         const uint4 *src = reinterpret_cast<const uint4 *>(dsec + 256 + (SUMMED ? decode_table_bytes(s.K) : 0)) +
                            (size_t)slice * s.K * CH;
         uint4 *dst = reinterpret_cast<uint4 *>(table);
-        if (SPLIT) {
+        if (F32) {
+            // entry (code j, stage r) = channels 4 slice .. 4 slice + 3 of codeword j of stage r
+            for (uint32_t t = tid; t < (uint32_t)s.K * 8; t += kDecThreads) {
+                const uint32_t r = t & 7u, j = t >> 3;
+                dst[t] = __ldg(reinterpret_cast<const uint4 *>(cb + ((size_t)r * s.K + j) * 32) + slice);
+            }
+        } else if (SPLIT) {
             // entry (code, stage) = elements 4 slice .. + 3 (half of the entry of slice / 2 in the prepared
             // table) followed by their partners 16 elements on (the same half of the entry of slice / 2 + 2)
             const uint2 *half = reinterpret_cast<const uint2 *>(dsec + 256 + (SUMMED ? decode_table_bytes(s.K) : 0));
@@ -644,6 +654,7 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
         // integer sums of level * scale: one 16-bit x 8-bit dot-product instruction per channel and stage,
         // or (summed levels) plain additions of the table words and two such instructions per channel
         uint32_t acc[CH], even[CH / 2], odd[CH / 2];
+        float facc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
         for (int i = 0; i < CH; ++i) acc[i] = 0u;
 #pragma unroll
@@ -656,6 +667,12 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
             const uint32_t line = (k & 1) ? ((w >> (16 - kShift)) & (0xFFFFu << kShift)) : ((w << kShift) & (0xFFFFu << kShift));
             const uint32_t a = smem_table + (line | unit[k]);
             uint32_t e[CH / 2];
+            if (F32) {
+                float f0, f1, f2, f3;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(f0), "=f"(f1), "=f"(f2), "=f"(f3) : "r"(a));
+                facc[0] += f0; facc[1] += f1; facc[2] += f2; facc[3] += f3;
+                continue;
+            }
             if (CH == 8)
                 asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(e[0]), "=r"(e[1]), "=r"(e[CH / 2 - 2]), "=r"(e[CH / 2 - 1]) : "r"(a));
             else
@@ -683,9 +700,9 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
         {
             const float bs = base * sd, cs = bias * sd;
 #pragma unroll
-            for (int i = 0; i < CH; ++i) o8[i] = fmaf((float)acc[i], bs, cs);
+            for (int i = 0; i < CH; ++i) o8[i] = F32 ? facc[i & 3] * sd : fmaf((float)acc[i], bs, cs);
         }
-        if (fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
+        if (!F32 && fabsf(sd) > exact_above && fabsf(sd) < INFINITY) {
             // too coarse for this deviation: the float32 codewords themselves, summed in stage order
             float ex[CH];
 #pragma unroll
@@ -864,7 +881,9 @@ decode_quoted_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__
 {
     extern __shared__ __align__(128) uint8_t table[];
     const int kind = sample_table_kind(std16, n, dsec);
-    if (kind == 2)
+    if (kind == 2 && FCH == 4)
+        decode_levels_fast<DT, 4, LAYOUT, BITS, false, 0, true>(s, codes, std16, n, dsec, cb, out, stride, st, table);
+    else if (kind == 2)
         decode_sliced_body<DT, FCH, true>(s, codes, std16, n, dsec, cb, out, stride, st, table);
     else if (kind == 1)
         decode_levels_fast<DT, LCH, LAYOUT, BITS, false>(s, codes, std16, n, dsec, cb, out, stride, st, table);

@@ -215,6 +215,37 @@ def decode_rope(codes, std_bits, codebooks, positions, base=10000.0, style=ROPE_
     return out if out_dtype is None else round_to(out, out_dtype)
 
 
+def attention_decode(q, codes_k, std_bits_k, codes_v, std_bits_v, codebooks_k, codebooks_v, kv_heads, scale,
+                     positions=None, base=10000.0, style=ROPE_HALVES, dim=128, layout_k=CONTIGUOUS,
+                     layout_v=CONTIGUOUS):
+    """One new token attending over a compressed cache (Section 1: the cache is what
+    long-context decoding loads; Section 3: keys are stored before the rotary
+    embedding, so they are rotated as they are read; Section 2.2: a cached vector is
+    the sum of its codewords times its deviation).  Rows of the cache are
+    [token][kv head]; query head i reads kv head i // (query heads / kv heads).  For
+    every query head: scores s_t = scale * q . k_t over the tokens, weights
+    softmax(s), output sum_t w_t v_t.  ``positions`` None leaves the keys unrotated.
+    The paper gives no formula for this step: it is the usual scaled dot-product
+    attention of the models it quantizes.  q [Hq][dim]; returns float64 [Hq][dim]."""
+    q = _f64(q)
+    n = len(codes_k)
+    T = n // kv_heads
+    k = decode(codes_k, std_bits_k, codebooks_k, dim, layout_k)
+    if positions is not None:
+        k = rope(k, np.repeat(np.asarray(positions), kv_heads), base, style)
+    v = decode(codes_v, std_bits_v, codebooks_v, dim, layout_v)
+    k, v = k.reshape(T, kv_heads, dim), v.reshape(T, kv_heads, dim)
+    per = q.shape[0] // kv_heads
+    out = np.zeros((q.shape[0], dim))
+    for i in range(q.shape[0]):
+        h = i // per
+        s = scale * (k[:, h, :] @ q[i])
+        w = np.exp(s - s.max())
+        w /= w.sum()
+        out[i] = w @ v[:, h, :]
+    return out
+
+
 def learn_step(x, codebooks, ema_count, ema_sum, decay, eps, group_dim=32, layout=CONTIGUOUS, ddof=0):
     """One codebook-learning step (Section 3): the batch is encoded with the
     current codebooks and these assignments feed the EMA update."""

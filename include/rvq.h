@@ -231,6 +231,44 @@ int rvq_rope_table(int32_t dim, double base, int32_t positions, float *cos_sin /
                    void *stream /* cudaStream_t */);
 
 /*
+ * Attention of one new token over a compressed cache, without the decoded keys
+ * and values ever reaching global memory (Section 1: loading the cache is what
+ * bounds decoding at long context; Section 3: keys are quantized before the rotary
+ * embedding, so they are rotated as they are read; Section 2.2: a cached vector is
+ * std * sum of its codewords).  The paper gives no formula for this step; it is the
+ * scaled dot-product attention of the models it quantizes.  Cache rows are
+ * [token][kv head] (row t * kv_heads + h); query head i reads kv head
+ * i / (q_heads / kv_heads).  With k^_t, v^_t the decoded head vectors of token t
+ * (float32 sums, keys rotated as under rvq_decode_rope with pairing and cos_sin):
+ *   s_t = scale * q_i . k^_t ;  w = softmax_t(s) ;  out_i = sum_t w_t v^_t.
+ *   cfg_k, cfg_v   in   host: the two quantizers (dim 128, groups of 32, depth <= 8,
+ *                       at most 1792 codes per stage; layouts and code widths may differ;
+ *                       x_dtype is not used)
+ *   q              in   device float32 [q_heads][128], already rotated to its own position
+ *   codes_k, std_k, codes_v, std_v   in   as produced by rvq_encode, tokens * kv_heads rows
+ *   tokens         in   >= 1
+ *   kv_heads       in   8;  q_heads 8, 16 or 32
+ *   position       in   device int32 [tokens], or NULL: token t sits at position t
+ *                       (values outside [0, positions) are clamped into it)
+ *   cos_sin        in   device float32 [positions][64][2] (rvq_rope_table), or NULL:
+ *                       the keys are used as stored
+ *   out            out  device float32 [q_heads][128]
+ *   workspace           rvq_attention_workspace_bytes(tokens, q_heads) bytes, 256-byte aligned
+ * Arithmetic: float32 codeword tables in shared memory (exact float32 sums), float32
+ * dot products and weights; the order of the float32 sums over tokens and channel
+ * slices is not fixed (reductions in global memory).  Codes >= K are read as code 0
+ * and counted in status->bad_codes.  Other shapes: RVQ_ERR_UNSUPPORTED.
+ */
+size_t rvq_attention_workspace_bytes(int64_t tokens, int32_t q_heads);
+int rvq_attention_decode(const rvq_config *cfg_k /* host */, const rvq_config *cfg_v /* host */,
+                         const float *q, int32_t q_heads, const void *codes_k, const uint16_t *std_k,
+                         const void *codes_v, const uint16_t *std_v, int64_t tokens, int32_t kv_heads,
+                         const float *codebooks_k, const float *codebooks_v, const int32_t *position,
+                         const float *cos_sin, int32_t positions, int32_t pairing, float scale,
+                         float *out, void *workspace, size_t workspace_bytes, rvq_status *status,
+                         void *stream /* cudaStream_t */);
+
+/*
  * One EMA codebook update (Section 3: the codebooks follow an exponential moving
  * average with decay 0.99; Section 2.1: EMA in place of the
  * codebook loss).  With n_r[j] the number of group rows whose stage-r code is j

@@ -81,6 +81,11 @@ def _load() -> ctypes.CDLL:
     lib.rvq_decode_rope.restype = ctypes.c_int
     lib.rvq_decode_rope.argtypes = [cfgp, vp, vp, i64, vp, vp, vp, ctypes.c_int32, vp, ctypes.c_int32,
                                     ctypes.c_int32, vp, i64, vp, vp]
+    lib.rvq_attention_workspace_bytes.restype = sz
+    lib.rvq_attention_workspace_bytes.argtypes = [i64, ctypes.c_int32]
+    lib.rvq_attention_decode.restype = ctypes.c_int
+    lib.rvq_attention_decode.argtypes = [cfgp, cfgp, vp, ctypes.c_int32, vp, vp, vp, vp, i64, ctypes.c_int32, vp, vp,
+                                         vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, vp, vp, sz, vp, vp]
     lib.rvq_learn_step.restype = ctypes.c_int
     lib.rvq_learn_step.argtypes = [cfgp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float,
                                    vp, sz, vp, vp]
@@ -93,7 +98,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 
-EXPORTS = ("rvq_selftest_encode_timeout", "rvq_rope_table", "rvq_decode_rope", "rvq_learn_step", "rvq_kmeans_workspace_bytes", "rvq_kmeans_init", "rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
+EXPORTS = ("rvq_attention_workspace_bytes", "rvq_attention_decode", "rvq_selftest_encode_timeout", "rvq_rope_table", "rvq_decode_rope", "rvq_learn_step", "rvq_kmeans_workspace_bytes", "rvq_kmeans_init", "rvq_encode_stats", "rvq_ema_update_static", "rvq_ema_static_scratch_bytes", "rvq_encode_exact", "rvq_status_string", "rvq_version", "rvq_launch_count", "rvq_ema_stats", "rvq_ema_apply", "rvq_code_bytes", "rvq_prepared_bytes",
            "rvq_prepare_codebooks", "rvq_workspace_bytes", "rvq_encode", "rvq_decode",
            "rvq_ema_update")
 
@@ -259,6 +264,23 @@ def rvq_decode_rope(cfg, codes, std_f16, n, codebooks, prepared, position, vecto
                              _ptr(status), _stream(stream))
     if check:
         _check(rc, "rvq_decode_rope")
+    return rc
+
+
+def rvq_attention_workspace_bytes(tokens: int, q_heads: int) -> int:
+    return int(lib.rvq_attention_workspace_bytes(tokens, q_heads))
+
+
+def rvq_attention_decode(cfg_k, cfg_v, q, q_heads, codes_k, std_k, codes_v, std_v, tokens, kv_heads, codebooks_k,
+                         codebooks_v, position, cos_sin, positions, pairing, scale, out, workspace, workspace_bytes,
+                         status=None, stream=None, check=True) -> int:
+    """out = attention of the query heads q over the compressed cache (keys rotated as they are read)."""
+    rc = lib.rvq_attention_decode(ctypes.byref(cfg_k), ctypes.byref(cfg_v), _ptr(q), q_heads, _ptr(codes_k), _ptr(std_k),
+                                  _ptr(codes_v), _ptr(std_v), tokens, kv_heads, _ptr(codebooks_k), _ptr(codebooks_v),
+                                  _ptr(position), _ptr(cos_sin), positions, pairing, scale, _ptr(out), _ptr(workspace),
+                                  workspace_bytes, _ptr(status), _stream(stream))
+    if check:
+        _check(rc, "rvq_attention_decode")
     return rc
 
 

@@ -229,6 +229,37 @@ int rvq_decode_rope(const rvq_config *cfg, const void *codes, const uint16_t *st
                               pairing, x_out, out_row_stride, status, (cudaStream_t)stream);
 }
 
+size_t rvq_attention_workspace_bytes(int64_t tokens, int32_t q_heads)
+{
+    if (tokens < 1 || q_heads < 1 || q_heads > 32) return 0;
+    return attention_workspace_bytes(tokens, q_heads);
+}
+
+int rvq_attention_decode(const rvq_config *cfg_k, const rvq_config *cfg_v, const float *q, int32_t q_heads,
+                         const void *codes_k, const uint16_t *std_k, const void *codes_v, const uint16_t *std_v,
+                         int64_t tokens, int32_t kv_heads, const float *codebooks_k, const float *codebooks_v,
+                         const int32_t *position, const float *cos_sin, int32_t positions, int32_t pairing,
+                         float scale, float *out, void *workspace, size_t workspace_bytes, rvq_status *status,
+                         void *stream)
+{
+    Shape sk, sv;
+    int rc = make_shape(cfg_k, &sk);
+    if (rc != RVQ_OK) return rc;
+    if ((rc = make_shape(cfg_v, &sv)) != RVQ_OK) return rc;
+    if (!q || !codes_k || !std_k || !codes_v || !std_v || !codebooks_k || !codebooks_v || !out || !workspace)
+        return RVQ_ERR_BADARG;
+    if (tokens < 1 || q_heads < 1 || kv_heads < 1 || !(scale == scale)) return RVQ_ERR_BADARG;
+    if (cos_sin && (positions < 1 || (pairing != RVQ_ROPE_HALVES && pairing != RVQ_ROPE_ADJACENT))) return RVQ_ERR_BADARG;
+    if (!attention_supported(sk, sv, kv_heads, q_heads)) return RVQ_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(codes_k) || !aligned16(codes_v) || !aligned16(codebooks_k) || !aligned16(codebooks_v) ||
+        !aligned16(cos_sin) || !aligned16(out) || !aligned256(workspace))
+        return RVQ_ERR_ALIGN;
+    if (workspace_bytes < attention_workspace_bytes(tokens, q_heads)) return RVQ_ERR_WORKSPACE;
+    return launch_attention_decode(sk, sv, q, q_heads, codes_k, std_k, codes_v, std_v, tokens, codebooks_k, codebooks_v,
+                                   position, cos_sin, positions, pairing, scale, out, workspace, status,
+                                   (cudaStream_t)stream);
+}
+
 static int check_ema_common(const Shape &s, const void *x, int64_t n, int64_t stride, const void *codes,
                             const float *codebooks)
 {

@@ -64,20 +64,23 @@ __device__ __forceinline__ void att_fill_table(const Shape &s, const float *__re
 struct AttRow {
     uint32_t c0, c1, c2, c3;
     uint16_t sd;
-    int pos;
 };
+// Position of a token: the caller's, or the token's index.
+__device__ __forceinline__ int att_position(const int32_t *__restrict__ position, int64_t token, int64_t tokens)
+{
+    if (token >= tokens) return 0;
+    return position ? __ldg(position + token) : (int)(token < 0x7FFFFFFF ? token : 0x7FFFFFFF);
+}
 __device__ __forceinline__ void att_fetch(const Shape &s, const void *__restrict__ codes,
-                                          const uint16_t *__restrict__ std16, const int32_t *__restrict__ position,
-                                          int64_t token, int64_t tokens, int lane, AttRow &a)
+                                          const uint16_t *__restrict__ std16, int64_t token, int64_t tokens, int lane,
+                                          AttRow &a)
 {
     a.c0 = a.c1 = a.c2 = a.c3 = 0u;
     a.sd = 0;
-    a.pos = 0;
     if (token >= tokens) return;
     const int64_t v = token * 8 + (lane >> 2);
     const int g = lane & 3;
     a.sd = __ldg(std16 + v);
-    a.pos = position ? __ldg(position + token) : (int)(token < 0x7FFFFFFF ? token : 0x7FFFFFFF);
     if (s.bits == 16 && s.R == 8) {
         const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + (v * 4 + g));
         a.c0 = c.x; a.c1 = c.y; a.c2 = c.z; a.c3 = c.w;
@@ -131,6 +134,37 @@ __device__ __forceinline__ void att_gather(const AttRow &a, uint32_t K, uint32_t
     }
 }
 
+// (cos, sin) of the rotary pairs of this thread's four channels at position `pos`:
+// c[i], s[i] belong to place i (half-split pairs on strided groups and adjacent pairs on
+// contiguous groups have two pairs in the thread: places 0 and 1 of c, s).
+template <int LAYOUT, int ROPE>
+__device__ __forceinline__ void att_cos_sin(const float2 *__restrict__ cos_sin, int positions, int pos, int sl, int g,
+                                            float (&c)[4], float (&sn)[4])
+{
+    c[0] = c[1] = c[2] = c[3] = 1.0f;
+    sn[0] = sn[1] = sn[2] = sn[3] = 0.0f;
+    if (ROPE == 0) return;
+    const float2 *cs = cos_sin + (size_t)min(max(pos, 0), positions - 1) * 64;
+    if (ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED) {
+        // places (0, 2) and (1, 3): channels 4 (2 sl + i) + g and 64 further on; that channel is the pair
+#pragma unroll
+        for (int i = 0; i < 2; ++i) { const float2 t = __ldg(cs + 4 * (2 * sl + i) + g); c[i] = t.x; sn[i] = t.y; }
+    } else if (ROPE == 2 && LAYOUT == RVQ_GROUP_CONTIGUOUS) {
+        // channels 32 g + 4 sl + i: pairs 16 g + 2 sl + i / 2, both halves in the thread
+        const float4 t = __ldg(reinterpret_cast<const float4 *>(cs + 16 * g + 2 * sl));
+        c[0] = t.x; sn[0] = t.y; c[1] = t.z; sn[1] = t.w;
+    } else if (ROPE == 1) {
+        // contiguous groups: channel 32 g + 4 sl + i and its partner in group g ^ 2; pairs 32 (g & 1) + 4 sl + i
+        const float4 *p = reinterpret_cast<const float4 *>(cs + 32 * (g & 1) + 4 * sl);
+        const float4 a = __ldg(p), b = __ldg(p + 1);
+        c[0] = a.x; sn[0] = a.y; c[1] = a.z; sn[1] = a.w; c[2] = b.x; sn[2] = b.y; c[3] = b.z; sn[3] = b.w;
+    } else {
+        // strided groups, pairs (2k, 2k + 1): channels 4 e + g and 4 e + (g ^ 1), e = 4 sl + i; pair 2 e + g / 2
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { const float2 t = __ldg(cs + 2 * (4 * sl + i) + (g >> 1)); c[i] = t.x; sn[i] = t.y; }
+    }
+}
+
 // Step 1.  ROPE 0: keys as stored; 1: pairs (k, k + 64); 2: pairs (2k, 2k + 1).
 template <int LAYOUT, int ROPE, int J>
 __global__ void __launch_bounds__(kAttThreads, 1)
@@ -154,52 +188,51 @@ att_scores_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
     __syncthreads();
     const uint32_t smem_table = (uint32_t)__cvta_generic_to_shared(smem);
     uint32_t bad = 0;
+    // Loads run ahead of their use: the codes, the deviation and the (cos, sin) values of the next token
+    // are asked for while this one is gathered, and the position of the token after that (the address
+    // of the (cos, sin) values hangs on it).
+    const int64_t step = (int64_t)parts * 32, t0 = (int64_t)part * 32 + warp;
     AttRow next;
-    att_fetch(s, codes, std16, position, (int64_t)part * 32 + warp, tokens, lane, next);
-    for (int64_t t = (int64_t)part * 32 + warp; t < tokens; t += (int64_t)parts * 32) {
+    float cn[4], sn[4];
+    att_fetch(s, codes, std16, t0, tokens, lane, next);
+    att_cos_sin<LAYOUT, ROPE>(cos_sin, positions, att_position(position, t0, tokens), sl, g, cn, sn);
+    int pos_next = ROPE != 0 ? att_position(position, t0 + step, tokens) : 0;
+    for (int64_t t = t0; t < tokens; t += step) {
         const AttRow cur = next;
-        att_fetch(s, codes, std16, position, t + (int64_t)parts * 32, tokens, lane, next);
+        float cc[4], ss[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { cc[i] = cn[i]; ss[i] = sn[i]; }
+        att_cos_sin<LAYOUT, ROPE>(cos_sin, positions, pos_next, sl, g, cn, sn);
+        if (ROPE != 0) pos_next = att_position(position, t + 2 * step, tokens);
+        att_fetch(s, codes, std16, t + step, tokens, lane, next);
         float v[4];
         att_gather(cur, (uint32_t)s.K, (uint32_t)lane & 7u, smem_table, v, bad);
         const float sd = __half2float(__ushort_as_half(cur.sd));
 #pragma unroll
         for (int i = 0; i < 4; ++i) v[i] *= sd;
         if (ROPE != 0) {
-            const float2 *cs = cos_sin + (size_t)min(max(cur.pos, 0), positions - 1) * 64;
             if (ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED) {
-                // places (0, 2) and (1, 3): channels 4 (2 sl + i) + g and 64 further on; that channel is the pair
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
-                    const float2 c = __ldg(cs + 4 * (2 * sl + i) + g);
                     const float a = v[i], b = v[i + 2];
-                    v[i] = a * c.x - b * c.y;
-                    v[i + 2] = b * c.x + a * c.y;
+                    v[i] = a * cc[i] - b * ss[i];
+                    v[i + 2] = b * cc[i] + a * ss[i];
                 }
             } else if (ROPE == 2 && LAYOUT == RVQ_GROUP_CONTIGUOUS) {
-                // channels 32 g + 4 sl + i: pairs 16 g + 2 sl + i / 2, both halves here
-                const float4 c = __ldg(reinterpret_cast<const float4 *>(cs + 16 * g + 2 * sl));
-                const float a0 = v[0], b0 = v[1], a1 = v[2], b1 = v[3];
-                v[0] = a0 * c.x - b0 * c.y; v[1] = b0 * c.x + a0 * c.y;
-                v[2] = a1 * c.z - b1 * c.w; v[3] = b1 * c.z + a1 * c.w;
-            } else if (ROPE == 1) {
-                // contiguous groups: channel 32 g + 4 sl + i and its partner in group g ^ 2; pairs 32 (g & 1) + 4 sl + i
-                const float4 *p = reinterpret_cast<const float4 *>(cs + 32 * (g & 1) + 4 * sl);
-                const float4 ca = __ldg(p), cb2 = __ldg(p + 1);
-                const float cc[4] = {ca.x, ca.z, cb2.x, cb2.z}, ss[4] = {ca.y, ca.w, cb2.y, cb2.w};
-                const bool first = (g & 2) == 0;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float o = __shfl_xor_sync(0xFFFFFFFFu, v[i], 2);
-                    v[i] = first ? v[i] * cc[i] - o * ss[i] : v[i] * cc[i] + o * ss[i];
+                for (int i = 0; i < 2; ++i) {
+                    const float a = v[2 * i], b = v[2 * i + 1];
+                    v[2 * i] = a * cc[i] - b * ss[i];
+                    v[2 * i + 1] = b * cc[i] + a * ss[i];
                 }
             } else {
-                // strided groups, pairs (2k, 2k + 1): channels 4 e + g and 4 e + (g ^ 1), e = 4 sl + i; pair 2 e + g / 2
-                const bool first = (g & 1) == 0;
+                // the partner is the same place of group g ^ 2 (half-split pairs) or g ^ 1 (adjacent pairs)
+                const int other = ROPE == 1 ? 2 : 1;
+                const bool first = (g & other) == 0;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const float2 c = __ldg(cs + 2 * (4 * sl + i) + (g >> 1));
-                    const float o = __shfl_xor_sync(0xFFFFFFFFu, v[i], 1);
-                    v[i] = first ? v[i] * c.x - o * c.y : v[i] * c.x + o * c.y;
+                    const float o = __shfl_xor_sync(0xFFFFFFFFu, v[i], other);
+                    v[i] = first ? v[i] * cc[i] - o * ss[i] : v[i] * cc[i] + o * ss[i];
                 }
             }
         }
@@ -269,9 +302,8 @@ att_values_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
     // exp(scale s - m) = 2^(s * scale log2(e) - m log2(e))
     constexpr float kLog2e = 1.4426950408889634f;
     const float sl2 = scale * kLog2e;
-    float mneg[J];
-#pragma unroll
-    for (int j = 0; j < J; ++j) mneg[j] = -att_unordered(m_ord[h * J + j]) * kLog2e;
+    __shared__ float mneg_s[32];                             // -m log2(e) per query head (read back per token: registers are short)
+    if (threadIdx.x < 8 * J) mneg_s[threadIdx.x] = -att_unordered(m_ord[threadIdx.x]) * kLog2e;
     __syncthreads();
     const uint32_t smem_table = (uint32_t)__cvta_generic_to_shared(smem);
     uint32_t bad = 0;
@@ -279,7 +311,7 @@ att_values_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
 #pragma unroll
     for (int j = 0; j < J; ++j) { wsum[j] = 0.0f; acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.0f; }
     AttRow next;
-    att_fetch(s, codes, std16, nullptr, (int64_t)part * 32 + warp, tokens, lane, next);
+    att_fetch(s, codes, std16, (int64_t)part * 32 + warp, tokens, lane, next);
     for (int64_t t = (int64_t)part * 32 + warp; t < tokens; t += (int64_t)parts * 32) {
         const AttRow cur = next;
         // this token's scores, asked for before the gather
@@ -290,7 +322,7 @@ att_values_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
             else if (J == 2) { const float2 f = __ldg(reinterpret_cast<const float2 *>(src)); sc[0] = f.x; sc[J - 1] = f.y; }
             else sc[0] = __ldg(src);
         }
-        att_fetch(s, codes, std16, nullptr, t + (int64_t)parts * 32, tokens, lane, next);
+        att_fetch(s, codes, std16, t + (int64_t)parts * 32, tokens, lane, next);
         float v[4];
         att_gather(cur, (uint32_t)s.K, (uint32_t)lane & 7u, smem_table, v, bad);
         const float sd = __half2float(__ushort_as_half(cur.sd));
@@ -298,7 +330,7 @@ att_values_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
         for (int i = 0; i < 4; ++i) v[i] *= sd;
 #pragma unroll
         for (int j = 0; j < J; ++j) {
-            const float w = exp2f(fmaf(sc[j], sl2, mneg[j]));
+            const float w = exp2f(fmaf(sc[j], sl2, mneg_s[h * J + j]));
             wsum[j] += w;
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[j][i] = fmaf(w, v[i], acc[j][i]);

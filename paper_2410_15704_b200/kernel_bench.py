@@ -4,6 +4,7 @@
   python paper_2410_15704_b200/kernel_bench.py encode key_cache:4096 value_cache:32768 tiny:4096
   python paper_2410_15704_b200/kernel_bench.py decode decode_bandwidth:131072
   python paper_2410_15704_b200/kernel_bench.py decode_rope decode_bandwidth:131072
+  python paper_2410_15704_b200/kernel_bench.py attention decode_bandwidth:131072
   python paper_2410_15704_b200/kernel_bench.py ema ema_learning:131072
   python paper_2410_15704_b200/kernel_bench.py learn_step ema_learning:131072
   python paper_2410_15704_b200/kernel_bench.py kmeans ema_learning:131072 --iterations 10
@@ -73,7 +74,7 @@ def config_of(w, bits=None):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "decode_rope", "ema",
+    ap.add_argument("kernel", choices=["encode", "encode_stats", "encode_exact", "decode", "decode_rope", "attention", "ema",
                                        "learn_step", "kmeans"])
     ap.add_argument("--iterations", type=int, default=10, help="Lloyd iterations per stage (kmeans)")
     ap.add_argument("--shape", default=None,
@@ -88,7 +89,9 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     for spec in args.cases:
-        if args.kernel in ("decode", "decode_rope") and spec.startswith("decode_bandwidth"):
+        if args.kernel == "attention":
+            runs = [make(spec, layout=1)]
+        elif args.kernel in ("decode", "decode_rope") and spec.startswith("decode_bandwidth"):
             runs = [make(spec, layout=0), make(spec, layout=1)]
         elif spec.startswith("ablation") and args.shape:
             f = [int(t) for t in args.shape.split(",")]
@@ -102,6 +105,34 @@ def main():
             code_b = (G * R * w.code_bits + 31) // 32 * 4
             line = {"kernel": args.kernel, "workload": name, "vectors": n, "dim": w.dim, "group_dim": gd, "K": K, "R": R,
                     "layout": "strided" if w.layout else "contiguous", "code_bits": w.code_bits}
+            if args.kernel == "attention":
+                # one new token (32 query heads, 8 kv heads) over a cache of n / 8 tokens: the workload's codes as
+                # keys on strided groups (half-split rotary pairs, position = token index), the same codes read as
+                # values on contiguous groups
+                tokens = n // 8
+                cfg_k = rvq.make_config(w.dim, gd, rvq_synth.STRIDED, R, K, w.code_bits, rvq.BF16, 0)
+                cfg_v = rvq.make_config(w.dim, gd, rvq_synth.CONTIGUOUS, R, K, w.code_bits, rvq.BF16, 0)
+                b = rvq.alloc_buffers(cfg_k, n, w.codebooks)
+                b.codes.view(torch.int16)[: n * G * R].copy_(
+                    torch.from_numpy(w.codes.astype(np.uint16).view(np.int16).reshape(-1)))
+                b.std.copy_(torch.from_numpy(w.std_bits.view(np.int16)))
+                q = torch.from_numpy(np.random.default_rng(1).normal(size=(32, w.dim)).astype(np.float32)).cuda()
+                table = torch.empty(tokens, w.dim // 2, 2, device="cuda")
+                rvq.rvq_rope_table(w.dim, 500000.0, tokens, table)
+                ws_bytes = rvq.rvq_attention_workspace_bytes(tokens, 32)
+                ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+                out = torch.empty(32, w.dim, device="cuda")
+                med, best = timed(lambda: rvq.rvq_attention_decode(cfg_k, cfg_v, q, 32, b.codes, b.std, b.codes, b.std, tokens,
+                                                                   8, b.codebooks, b.codebooks, None, table, tokens,
+                                                                   rvq.ROPE_HALVES, float(w.dim) ** -0.5, out, ws, ws_bytes,
+                                                                   b.status), args.reps, flush)
+                nbytes = 2 * n * (code_b + 2) + tokens * (w.dim // 2) * 8          # both caches' codes and deviations, the table
+                line.update(tokens=tokens, ms_median=med, ms_best=best, cached_vectors_per_s=2 * n / med / 1e3, bytes=nbytes,
+                            GBps=nbytes / med / 1e6, frac_hbm=nbytes / med / 1e6 / hbm, peak=hbm, peak_source=src,
+                            decoded_bytes_never_written=2 * n * w.dim * 2)
+                line.update(rvq.read_status(b.status))
+                print(json.dumps(line), flush=True)
+                continue
             if args.kernel in ("decode", "decode_rope"):
                 cfg = config_of(w)
                 b = rvq.alloc_buffers(cfg, n, w.codebooks)

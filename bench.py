@@ -236,6 +236,33 @@ def side_workloads(torch, rvq, peaks, flush):
     out["decode_bandwidth"] = {"workload": "1048576 head vectors, uint16 codes uniform over 1024, fp16 std, bf16 out",
                                "headline": slow, **dec}
 
+    # the same codes as a cache of 131072 tokens x 8 kv heads: one new token (32 query heads) attends over it,
+    # keys on strided groups rotated at their token index, values on contiguous groups
+    w = rvq_synth.decode_bandwidth(layout=rvq_synth.STRIDED)
+    tokens = w.n // 8
+    cfg_k = rvq.make_config(w.dim, w.group_dim, rvq_synth.STRIDED, w.depth, w.codebook_size, 16, rvq.BF16, 0)
+    cfg_v = rvq.make_config(w.dim, w.group_dim, rvq_synth.CONTIGUOUS, w.depth, w.codebook_size, 16, rvq.BF16, 0)
+    b = rvq.alloc_buffers(cfg_k, w.n, w.codebooks)
+    b.codes.view(torch.int16)[: w.n * w.groups * w.depth].copy_(
+        torch.from_numpy(w.codes.astype(np.uint16).view(np.int16).reshape(-1)))
+    b.std.copy_(torch.from_numpy(w.std_bits.view(np.int16)))
+    q = torch.from_numpy(np.random.default_rng(1).normal(size=(32, w.dim)).astype(np.float32)).cuda()
+    table = torch.empty(tokens, w.dim // 2, 2, device="cuda")
+    rvq.rvq_rope_table(w.dim, 500000.0, tokens, table)
+    ws_bytes = rvq.rvq_attention_workspace_bytes(tokens, 32)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    att_out = torch.empty(32, w.dim, device="cuda")
+    med, best = time_launches(torch, lambda: rvq.rvq_attention_decode(
+        cfg_k, cfg_v, q, 32, b.codes, b.std, b.codes, b.std, tokens, 8, b.codebooks, b.codebooks, None, table, tokens,
+        rvq.ROPE_HALVES, float(w.dim) ** -0.5, att_out, ws, ws_bytes, b.status), flush)
+    att_bytes = 2 * w.n * (64 + 2) + tokens * (w.dim // 2) * 8
+    out["attention_over_cache"] = {"workload": "one token, 32 query heads, over 131072 cached tokens x 8 kv heads "
+                                               "(2 x 1048576 compressed head vectors, K=1024, R=8), rotary keys",
+                                   "ms": med, "ms_best": best, "cached_Mvectors/s": 2 * w.n / med / 1e3,
+                                   "GB/s": att_bytes / med / 1e6, "frac_hbm": att_bytes / med / 1e6 / hbm,
+                                   "bytes": att_bytes, "decoded_bytes_never_written": 2 * w.n * w.dim * 2}
+    del b, ws, table
+
     # value cache: 2048 codes per stage, 11-bit packed codes, contiguous groups
     w = rvq_synth.value_cache()
     cfg = rvq.make_config(w.dim, w.group_dim, w.layout, w.depth, w.codebook_size, w.code_bits, rvq.BF16, 0)

@@ -164,12 +164,8 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&u)[32
                  "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
                  : RVQ_OUT32(u) : "r"(taddr));
 }
-// Waits for every tcgen05.ld of this thread; the array passes through so that no
-// use of it can be scheduled ahead of the wait.
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&u)[32])
-{
-    asm volatile("tcgen05.wait::ld.sync.aligned;" : RVQ_INOUT32(u) : : "memory");
-}
+// Waits for every tcgen05.ld of this thread; the arrays pass through so that no
+// use of them can be scheduled ahead of the wait.
 __device__ __forceinline__ void tmem_ld_wait4(uint32_t (&u)[32], uint32_t (&v)[32], uint32_t (&w)[32], uint32_t (&x)[32])
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : RVQ_INOUT32(u) : : "memory");

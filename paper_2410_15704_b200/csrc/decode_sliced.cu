@@ -822,7 +822,8 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
     if (bad && st && slice == 0) atomicAdd(&st->bad_codes, bad);   // every slice sees the same codes
 }
 
-// True when more than an eighth of a sample of up to 256 deviations is beyond the level tables' reach.
+// True when more than one in 64 of a sample of up to 256 deviations is beyond the level tables' reach
+// (such a row takes the exact route and holds its whole warp up).
 // Uniform over the CTA (and over all CTAs of a launch: they read the same sample).
 __device__ __forceinline__ bool sample_wants_float32(const uint16_t *__restrict__ std16, int64_t n,
                                                   const uint8_t *__restrict__ dsec, float reach)
@@ -833,7 +834,7 @@ __device__ __forceinline__ bool sample_wants_float32(const uint16_t *__restrict_
     const bool beyond = threadIdx.x < samples &&
                         fabsf(__half2float(__ushort_as_half(std16[threadIdx.x * every]))) > exact_above;
     const int far = __syncthreads_count(beyond);
-    return (int64_t)far * 8 > samples;
+    return (int64_t)far * 64 > samples;
 }
 
 // PICK: with up to 1536 codes per stage and 16-bit outputs both kinds of table fit, and which one

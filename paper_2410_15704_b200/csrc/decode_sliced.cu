@@ -517,9 +517,11 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
                    const uint8_t *__restrict__ dsec, const float *__restrict__ cb, void *__restrict__ out,
                    int64_t stride, rvq_status *st, uint8_t *table, RopeArgs ra = RopeArgs())
 {
-    static_assert(ROPE == 0 || CH == 8, "the rotary variant uses 8-channel slices");
-    static_assert(!F32 || (CH == 4 && !SUMMED && ROPE == 0), "float32 tables: 4-channel slices, no rotation here");
-    constexpr bool SPLIT = ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED;   // slice = two runs of four elements
+    static_assert(ROPE == 0 || CH == 8 || F32, "the rotary variant uses 8-channel level slices or 4-channel float32 slices");
+    static_assert(!F32 || (CH == 4 && !SUMMED), "float32 tables: 4-channel slices");
+    // half-split pairs on strided groups: a slice is two runs of elements 16 apart (CH / 2 each), so that
+    // both channels of a pair are in the thread
+    constexpr bool SPLIT = ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED;
     constexpr int NS = 32 / CH;                                  // slices
     if ((int)blockIdx.x >= ((int)gridDim.x / NS) * NS) return;
     constexpr uint32_t kEntry = F32 ? 16 : 2 * CH;               // bytes per (code, stage); a code's line is 8 entries
@@ -532,10 +534,18 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
                            (size_t)slice * s.K * CH;
         uint4 *dst = reinterpret_cast<uint4 *>(table);
         if (F32) {
-            // entry (code j, stage r) = channels 4 slice .. 4 slice + 3 of codeword j of stage r
+            // entry (code j, stage r) = elements 4 slice .. 4 slice + 3 of codeword j of stage r (rotary slices
+            // of strided groups: 2 slice, 2 slice + 1 and the two 16 elements on)
             for (uint32_t t = tid; t < (uint32_t)s.K * 8; t += kDecThreads) {
                 const uint32_t r = t & 7u, j = t >> 3;
-                dst[t] = __ldg(reinterpret_cast<const uint4 *>(cb + ((size_t)r * s.K + j) * 32) + slice);
+                const float *src = cb + ((size_t)r * s.K + j) * 32;
+                if (SPLIT) {
+                    const uint2 a = __ldg(reinterpret_cast<const uint2 *>(src + 2 * slice));
+                    const uint2 b = __ldg(reinterpret_cast<const uint2 *>(src + 2 * slice + 16));
+                    dst[t] = make_uint4(a.x, a.y, b.x, b.y);
+                } else {
+                    dst[t] = __ldg(reinterpret_cast<const uint4 *>(src) + slice);
+                }
             }
         } else if (SPLIT) {
             // entry (code, stage) = elements 4 slice .. + 3 (half of the entry of slice / 2 in the prepared
@@ -612,9 +622,10 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
         const float2 *cs = nullptr;
         if (ROPE != 0) {
             cs = ra.table + (size_t)min(max(ppos, 0), ra.positions - 1) * 64;
-            const float2 *mine = ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED ? cs + 16 * slice
-                                 : ROPE == 2 && LAYOUT == RVQ_GROUP_CONTIGUOUS ? cs + g * 16 + slice * 4
-                                 : ROPE == 1 ? cs + (g & 1u) * 32 + slice * 8 : cs + 16 * slice;
+            // (pairs per slice: CH / 2 with both halves in the thread, CH otherwise)
+            const float2 *mine = ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED ? cs + 2 * CH * slice
+                                 : ROPE == 2 && LAYOUT == RVQ_GROUP_CONTIGUOUS ? cs + g * 16 + slice * (CH / 2)
+                                 : ROPE == 1 ? cs + (g & 1u) * 32 + slice * CH : cs + 2 * CH * slice;
             asm volatile("prefetch.global.L1 [%0];" ::"l"(mine));
         }
         fetch(row + parts * kDecThreads, p0, p1, p2, p3, psd, ppos);
@@ -722,7 +733,46 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
 #pragma unroll
             for (int i = 0; i < CH; ++i) o8[i] = ex[i] * sd;
         }
-        if (ROPE != 0) {
+        if (ROPE != 0 && F32) {
+            // four channels per thread: the same four cases as below at half the width
+            if (ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED) {
+                // places (0, 2) and (1, 3): channels 4 (2 slice + i) + g = pair index, and 64 further on
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float2 c = __ldg(cs + (2 * slice + i) * 4 + g);
+                    const float a = o8[i], b = o8[i + 2];
+                    o8[i] = a * c.x - b * c.y;
+                    o8[i + 2] = b * c.x + a * c.y;
+                }
+            } else if (ROPE == 2 && LAYOUT == RVQ_GROUP_CONTIGUOUS) {
+                // channels 32 g + 4 slice + i: pairs 16 g + 2 slice + i / 2
+                const float4 c = __ldg(reinterpret_cast<const float4 *>(cs + g * 16 + slice * 2));
+                const float a0 = o8[0], b0 = o8[1], a1 = o8[2], b1 = o8[3];
+                o8[0] = a0 * c.x - b0 * c.y; o8[1] = b0 * c.x + a0 * c.y;
+                o8[2] = a1 * c.z - b1 * c.w; o8[3] = b1 * c.z + a1 * c.w;
+            } else if (ROPE == 1) {
+                // contiguous groups: the partner is the same place of group g ^ 2; pairs 32 (g & 1) + 4 slice + i
+                const float4 *q = reinterpret_cast<const float4 *>(cs + (g & 1u) * 32 + slice * 4);
+                const bool first = (g & 2u) == 0;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float4 c = __ldg(q + h);
+                    const float p0 = __shfl_xor_sync(0xFFFFFFFFu, o8[2 * h], 2);
+                    const float p1 = __shfl_xor_sync(0xFFFFFFFFu, o8[2 * h + 1], 2);
+                    o8[2 * h] = first ? o8[2 * h] * c.x - p0 * c.y : o8[2 * h] * c.x + p0 * c.y;
+                    o8[2 * h + 1] = first ? o8[2 * h + 1] * c.z - p1 * c.w : o8[2 * h + 1] * c.z + p1 * c.w;
+                }
+            } else {
+                // strided groups, pairs (2k, 2k + 1): channels 4 e + g and 4 e + (g ^ 1), e = 4 slice + i; pair 2 e + g / 2
+                const bool first = (g & 1u) == 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 c = __ldg(cs + 2 * (4 * slice + i) + (g >> 1));
+                    const float p = __shfl_xor_sync(0xFFFFFFFFu, o8[i], 1);
+                    o8[i] = first ? o8[i] * c.x - p * c.y : o8[i] * c.x + p * c.y;
+                }
+            }
+        } else if (ROPE != 0) {
             // (cos, sin) of the pairs of this thread's channels
             if (ROPE == 1 && LAYOUT == RVQ_GROUP_STRIDED) {
                 // places 0..3 are channels 4 (4 slice + i) + g = pair index; places 4..7 their partners 64 on
@@ -772,7 +822,12 @@ decode_levels_fast(const Shape &s, const void *__restrict__ codes, const uint16_
 #pragma unroll
         for (int c = 0; c < CH / 2; ++c) w[c] = Out<DT>::pack(o8[2 * c], o8[2 * c + 1]);
         uint16_t *o16 = reinterpret_cast<uint16_t *>(out) + (size_t)v * stride;
-        if (SPLIT) {
+        if (SPLIT && F32) {
+            // the thread's places are elements 2 slice, 2 slice + 1 and their partners 16 on: lane L stores
+            // the four groups of place L
+            const uint2 t = transpose_group_elements(w[0], w[1], g);
+            if (live) *reinterpret_cast<uint2 *>(o16 + 4 * (2 * slice + (g & 1u) + 16 * (g >> 1))) = t;
+        } else if (SPLIT) {
             // lane L stores element 4 slice + L of the four groups, and its partner 16 elements on
             const uint2 lo = transpose_group_elements(w[0], w[1], g);
             const uint2 hi = transpose_group_elements(w[CH / 2 - 2], w[CH / 2 - 1], g);
@@ -904,7 +959,7 @@ decode_rope_quoted_kernel(Shape s, const void *__restrict__ codes, const uint16_
     extern __shared__ __align__(128) uint8_t table[];
     const int kind = sample_table_kind(std16, n, dsec, 0.6e-3f);
     if (kind == 2)
-        decode_sliced_body<DT, 4, true, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
+        decode_levels_fast<DT, 4, LAYOUT, BITS, false, ROPE, true>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
     else if (kind == 1)
         decode_levels_fast<DT, 8, LAYOUT, BITS, false, ROPE>(s, codes, std16, n, dsec, cb, out, stride, st, table, ra);
     else

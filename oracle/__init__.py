@@ -32,6 +32,14 @@ Parity status of each function against something other than itself
                         pairing), identity at position 0, norm preservation,
                         additivity in the position, the relative-position
                         property of the inner product
+  attention_decode      pinned: the library's scaled dot-product attention in
+                        float64 (grouped heads spelled out), a pure-Python brute
+                        force, one-token / identical-keys / dominant-token /
+                        zero-scale special cases, token permutation, kv-head
+                        isolation; the paper prints no formula for this step
+                        (it is the attention of the models it quantizes)
+  check_codes           near-tie verdicts pinned on hand-worked stages
+                        (tests/golden/check_codes_near_tie.txt)
 """
 from __future__ import annotations
 

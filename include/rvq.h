@@ -246,7 +246,7 @@ int rvq_rope_table(int32_t dim, double base, int32_t positions, float *cos_sin /
  *                       x_dtype is not used)
  *   q              in   device float32 [q_heads][128], already rotated to its own position
  *   codes_k, std_k, codes_v, std_v   in   as produced by rvq_encode, tokens * kv_heads rows
- *   tokens         in   >= 1
+ *   tokens         in   1 .. 2^26 - 4096
  *   kv_heads       in   8;  q_heads 8, 16 or 32
  *   position       in   device int32 [tokens], or NULL: token t sits at position t
  *                       (values outside [0, positions) are clamped into it)

@@ -250,7 +250,7 @@ int rvq_attention_decode(const rvq_config *cfg_k, const rvq_config *cfg_v, const
         return RVQ_ERR_BADARG;
     if (tokens < 1 || q_heads < 1 || kv_heads < 1 || !(scale == scale)) return RVQ_ERR_BADARG;
     if (cos_sin && (positions < 1 || (pairing != RVQ_ROPE_HALVES && pairing != RVQ_ROPE_ADJACENT))) return RVQ_ERR_BADARG;
-    if (!attention_supported(sk, sv, kv_heads, q_heads)) return RVQ_ERR_UNSUPPORTED;
+    if (!attention_supported(sk, sv, kv_heads, q_heads, tokens)) return RVQ_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(codes_k) || !aligned16(codes_v) || !aligned16(codebooks_k) || !aligned16(codebooks_v) ||
         !aligned16(cos_sin) || !aligned16(out) || !aligned256(workspace))
         return RVQ_ERR_ALIGN;

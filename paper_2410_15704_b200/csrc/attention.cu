@@ -66,26 +66,26 @@ struct AttRow {
     uint16_t sd;
 };
 // Position of a token: the caller's, or the token's index.
-__device__ __forceinline__ int att_position(const int32_t *__restrict__ position, int64_t token, int64_t tokens)
+__device__ __forceinline__ int att_position(const int32_t *__restrict__ position, uint32_t token, uint32_t tokens)
 {
     if (token >= tokens) return 0;
-    return position ? __ldg(position + token) : (int)(token < 0x7FFFFFFF ? token : 0x7FFFFFFF);
+    return position ? __ldg(position + token) : (int)token;
 }
 __device__ __forceinline__ void att_fetch(const Shape &s, const void *__restrict__ codes,
-                                          const uint16_t *__restrict__ std16, int64_t token, int64_t tokens, int lane,
+                                          const uint16_t *__restrict__ std16, uint32_t token, uint32_t tokens, int lane,
                                           AttRow &a)
 {
     a.c0 = a.c1 = a.c2 = a.c3 = 0u;
     a.sd = 0;
     if (token >= tokens) return;
-    const int64_t v = token * 8 + (lane >> 2);
+    const uint32_t v = token * 8u + (uint32_t)(lane >> 2);    // (the launcher keeps tokens * 32 below 2^31)
     const int g = lane & 3;
     a.sd = __ldg(std16 + v);
     if (s.bits == 16 && s.R == 8) {
-        const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + (v * 4 + g));
+        const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + (v * 4u + (uint32_t)g));
         a.c0 = c.x; a.c1 = c.y; a.c2 = c.z; a.c3 = c.w;
     } else {
-        const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + v * s.code_bytes;
+        const uint8_t *vec = reinterpret_cast<const uint8_t *>(codes) + (size_t)v * s.code_bytes;
         uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int r = 0; r < 8; ++r)
@@ -191,20 +191,20 @@ att_scores_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
     // Loads run ahead of their use: the codes, the deviation and the (cos, sin) values of the next token
     // are asked for while this one is gathered, and the position of the token after that (the address
     // of the (cos, sin) values hangs on it).
-    const int64_t step = (int64_t)parts * 32, t0 = (int64_t)part * 32 + warp;
+    const uint32_t T = (uint32_t)tokens, step = (uint32_t)parts * 32u, t0 = (uint32_t)part * 32u + (uint32_t)warp;
     AttRow next;
     float cn[4], sn[4];
-    att_fetch(s, codes, std16, t0, tokens, lane, next);
-    att_cos_sin<LAYOUT, ROPE>(cos_sin, positions, att_position(position, t0, tokens), sl, g, cn, sn);
-    int pos_next = ROPE != 0 ? att_position(position, t0 + step, tokens) : 0;
-    for (int64_t t = t0; t < tokens; t += step) {
+    att_fetch(s, codes, std16, t0, T, lane, next);
+    att_cos_sin<LAYOUT, ROPE>(cos_sin, positions, att_position(position, t0, T), sl, g, cn, sn);
+    int pos_next = ROPE != 0 ? att_position(position, t0 + step, T) : 0;
+    for (uint32_t t = t0; t < T; t += step) {
         const AttRow cur = next;
         float cc[4], ss[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) { cc[i] = cn[i]; ss[i] = sn[i]; }
         att_cos_sin<LAYOUT, ROPE>(cos_sin, positions, pos_next, sl, g, cn, sn);
-        if (ROPE != 0) pos_next = att_position(position, t + 2 * step, tokens);
-        att_fetch(s, codes, std16, t + step, tokens, lane, next);
+        if (ROPE != 0) pos_next = att_position(position, t + 2 * step, T);
+        att_fetch(s, codes, std16, t + step, T, lane, next);
         float v[4];
         att_gather(cur, (uint32_t)s.K, (uint32_t)lane & 7u, smem_table, v, bad);
         const float sd = __half2float(__ushort_as_half(cur.sd));
@@ -248,7 +248,7 @@ att_scores_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
             part_s[j] = a;
         }
         if (g == 0) {
-            float *dst = scores + ((size_t)t * 8 + h) * J;
+            float *dst = scores + (size_t)(t * 8u + (uint32_t)h) * J;
             if (J == 4) atomicAdd(reinterpret_cast<float4 *>(dst), make_float4(part_s[0], part_s[1], part_s[J - 2], part_s[J - 1]));
             else if (J == 2) atomicAdd(reinterpret_cast<float2 *>(dst), make_float2(part_s[0], part_s[J - 1]));
             else atomicAdd(dst, part_s[0]);
@@ -310,19 +310,20 @@ att_values_kernel(Shape s, const void *__restrict__ codes, const uint16_t *__res
     float acc[J][4], wsum[J];
 #pragma unroll
     for (int j = 0; j < J; ++j) { wsum[j] = 0.0f; acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.0f; }
+    const uint32_t T = (uint32_t)tokens, step = (uint32_t)parts * 32u;
     AttRow next;
-    att_fetch(s, codes, std16, (int64_t)part * 32 + warp, tokens, lane, next);
-    for (int64_t t = (int64_t)part * 32 + warp; t < tokens; t += (int64_t)parts * 32) {
+    att_fetch(s, codes, std16, (uint32_t)part * 32u + (uint32_t)warp, T, lane, next);
+    for (uint32_t t = (uint32_t)part * 32u + (uint32_t)warp; t < T; t += step) {
         const AttRow cur = next;
         // this token's scores, asked for before the gather
         float sc[J];
         {
-            const float *src = scores + ((size_t)t * 8 + h) * J;
+            const float *src = scores + (size_t)(t * 8u + (uint32_t)h) * J;
             if (J == 4) { const float4 f = __ldg(reinterpret_cast<const float4 *>(src)); sc[0] = f.x; sc[1] = f.y; sc[J - 2] = f.z; sc[J - 1] = f.w; }
             else if (J == 2) { const float2 f = __ldg(reinterpret_cast<const float2 *>(src)); sc[0] = f.x; sc[J - 1] = f.y; }
             else sc[0] = __ldg(src);
         }
-        att_fetch(s, codes, std16, t + (int64_t)parts * 32, tokens, lane, next);
+        att_fetch(s, codes, std16, t + step, T, lane, next);
         float v[4];
         att_gather(cur, (uint32_t)s.K, (uint32_t)lane & 7u, smem_table, v, bad);
         const float sd = __half2float(__ushort_as_half(cur.sd));
@@ -370,11 +371,16 @@ __global__ void att_finish_kernel(const float *__restrict__ out_acc, const float
 
 }  // namespace
 
-bool attention_supported(const Shape &sk, const Shape &sv, int kv_heads, int q_heads)
+// (token counts: the kernels index group rows, 32 per token, with 32-bit integers, and step past the end
+// by up to two strides of at most 18 * 32 tokens)
+constexpr int64_t kAttMaxTokens = (1LL << 26) - 4096;
+
+bool attention_supported(const Shape &sk, const Shape &sv, int kv_heads, int q_heads, int64_t tokens)
 {
     auto ok = [](const Shape &s) { return s.dim == 128 && s.gd == 32 && s.R <= 8 && s.K <= kAttMaxK; };
     const int J = kv_heads > 0 ? q_heads / kv_heads : 0;
-    return ok(sk) && ok(sv) && kv_heads == 8 && q_heads == kv_heads * J && (J == 1 || J == 2 || J == 4);
+    return ok(sk) && ok(sv) && kv_heads == 8 && q_heads == kv_heads * J && (J == 1 || J == 2 || J == 4) &&
+           tokens <= kAttMaxTokens;
 }
 
 size_t attention_workspace_bytes(int64_t tokens, int q_heads)

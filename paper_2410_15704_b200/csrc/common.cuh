@@ -57,7 +57,7 @@ size_t kmeans_workspace_bytes(const Shape &s, int64_t n);
 int launch_kmeans(const Shape &s, const void *x, int64_t n, int64_t stride, const int64_t *seed_rows,
                   int iterations, float *codebooks, void *prepared, void *workspace, rvq_status *st,
                   cudaStream_t stream);
-bool attention_supported(const Shape &sk, const Shape &sv, int kv_heads, int q_heads);
+bool attention_supported(const Shape &sk, const Shape &sv, int kv_heads, int q_heads, int64_t tokens);
 size_t attention_workspace_bytes(int64_t tokens, int q_heads);
 int launch_attention_decode(const Shape &sk, const Shape &sv, const float *q, int q_heads, const void *codes_k,
                             const uint16_t *std_k, const void *codes_v, const uint16_t *std_v, int64_t tokens,

@@ -162,7 +162,7 @@ int rvq_encode_stats(const rvq_config *cfg, const void *x, int64_t n, int64_t x_
     rc = encode_common(cfg, x, n, x_row_stride, codebooks, prepared, codes, std_f16, stage_energy, status, stream, true,
                        cnt, batch_sum);
     if (rc != RVQ_OK) return rc;
-    return launch_counts_to_float(cnt, batch_count, bins, st);
+    return launch_stats_finish(s, cnt, codebooks, batch_sum, batch_count, encode_tensor_deferred_stages(s), st);
 }
 
 int rvq_selftest_encode_timeout(const rvq_config *cfg, const void *x, int64_t n, int64_t x_row_stride,

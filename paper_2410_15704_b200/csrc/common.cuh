@@ -36,6 +36,10 @@ int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t strid
                          cudaStream_t stream, uint32_t *stat_cnt = nullptr, float *stat_sum = nullptr,
                          float *energy = nullptr, uint32_t wait_limit = 0, int drop_last_chain = 0);
 int launch_counts_to_float(const uint32_t *cnt, float *out, int bins, cudaStream_t stream);
+int encode_tensor_deferred_stages(const Shape &s);
+// counts to float32, and sum += count * codeword for the first `deferred` stages (see encode_tensor.cu)
+int launch_stats_finish(const Shape &s, const uint32_t *cnt, const float *cb, float *batch_sum, float *batch_count,
+                        int deferred, cudaStream_t stream);
 int launch_decode_gather(const Shape &s, const void *codes, const uint16_t *std16, int64_t n,
                          const float *cb, void *out, int64_t stride, rvq_status *st,
                          cudaStream_t stream);

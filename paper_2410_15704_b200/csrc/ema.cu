@@ -299,6 +299,28 @@ int launch_ema_stats(const Shape &s, const void *x, int64_t n, int64_t stride, c
     return check_launch();
 }
 
+// One thread per (bin, channel): the float32 count of the bin, and for the stages whose fused sums
+// were taken after the subtraction of the codeword, the codeword's share back: sum += count * C.
+__global__ void __launch_bounds__(256)
+stats_finish_kernel(const uint32_t *__restrict__ cnt, const float *__restrict__ cb, float *__restrict__ sum,
+                    float *__restrict__ out_count, int bins, int gd, int deferred_bins)
+{
+    const int t = blockIdx.x * 256 + threadIdx.x;
+    if (t >= bins * gd) return;
+    const int bin = t / gd, ch = t - bin * gd;
+    const float c = (float)cnt[bin];
+    if (ch == 0) out_count[bin] = c;
+    if (bin < deferred_bins) sum[t] = fmaf(c, cb[t], sum[t]);
+}
+
+int launch_stats_finish(const Shape &s, const uint32_t *cnt, const float *cb, float *batch_sum, float *batch_count,
+                        int deferred, cudaStream_t stream)
+{
+    const int bins = s.R * s.K, total = bins * s.gd;
+    stats_finish_kernel<<<(total + 255) / 256, 256, 0, stream>>>(cnt, cb, batch_sum, batch_count, bins, s.gd, deferred * s.K);
+    return check_launch();
+}
+
 int launch_counts_to_float(const uint32_t *cnt, float *out, int bins, cudaStream_t stream)
 {
     counts_to_float_kernel<<<(bins + 255) / 256, 256, 0, stream>>>(cnt, out, bins);

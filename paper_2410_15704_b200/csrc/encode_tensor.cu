@@ -61,7 +61,9 @@ constexpr int kOffListV = kOffZ + 32 * kRowsPerPass * 4;
 constexpr int kOffListI = kOffListV + (kListCap + 1) * kRowsPerPass * 4;   
 constexpr int kOffCodes = kOffListI + (kListCap + 1) * kRowsPerPass * 2;   
 constexpr int kOffBars = kOffCodes + kRowsPerPass * 16 * 2;          
-constexpr int kSmemBytes = kOffBars + 256;
+constexpr int kOffFlags = kOffBars + 256;                             // per row of the round: bit 0 valid, bit 1 degenerate
+constexpr int kSmemBytes = kOffFlags + 512;
+constexpr int kDeferMinSlots = 5;                                     // chunks a stage needs for its issuers to take the statistics
 
 // barrier slots
 constexpr int kBarFull = 0, kBarEmpty = kRing, kBarAReady = 2 * kRing, kBarAccFull = 2 * kRing + kTiles,
@@ -291,6 +293,7 @@ struct Params {
     float *energy;      // optional [R]: sum over the rows of the squared norm of what each stage leaves
     uint32_t wait_limit;   // polls after which a wait gives up (kWaitLimit; smaller only in the timeout self-test)
     int drop_last_chain;   // timeout self-test: 1 = tile 0's issuer leaves out the CTA's very last chain; else 0
+    int defer_stats;       // 1 = the statistics of every stage but the last are added by the MMA issuer warps (below)
 };
 
 // The tiles of one CTA: a contiguous run, done in `rounds` rounds of nearly equal size (<= kTiles).
@@ -395,8 +398,18 @@ encode_tensor_kernel(const Params p)
             const uint32_t acc = tmem + t * kTileCols, a0 = acc + 128;
             const uint32_t bar_ready = BAR(kBarAReady + t), bar_free = BAR(kBarAccFree + t), bar_acc = BAR(kBarAccFull + t);
             const uint32_t per_round = (uint32_t)s.R * (uint32_t)S;
-            uint32_t slot = 0, full_par = 0, s_in = 0, ready_par = 0, free_par = 1, in_round = 0;
+            uint32_t slot = 0, full_par = 0, s_in = 0, ready_par = 0, free_par = 1, in_round = 0, stage = 0;
             int round = 0;
+            // Deferred statistics (Section 3's EMA sums): while stage r+1 is swept, its input z_{r+1} -- what stage r
+            // left -- sits parked in shared memory, and this warp, idle between two chains, adds it to the bins of
+            // the stage-r codes, one group of 32 rows after each of the chains 1..4 of the stage.  The sum of a
+            // bin's stage-r INPUTS is that plus count * codeword (z_r = z_{r+1} + C_r[j]), which the caller adds
+            // afterwards.  Ordering: the epilogue parks z_{r+1} and has written the stage-r codes before it hands
+            // chunk 0's accumulator back, which this warp has waited for before chain 1; and it cannot finish the
+            // stage, and park anew, before the chains that this warp issues after the additions.
+            const float *zp = reinterpret_cast<const float *>(smem + kOffZ);
+            const uint16_t *codes_s = reinterpret_cast<const uint16_t *>(smem + kOffCodes);
+            const uint8_t *flags_s = smem + kOffFlags;
             bool ok = true, first = true, active = t < work.round_size(0);
             for (uint32_t q = 0; q < total && ok; ++q) {
                 ok = mbar_wait(BAR(kBarFull + slot), full_par, abort_flag);
@@ -406,7 +419,7 @@ encode_tensor_kernel(const Params p)
                     if (ok && lane == 0) mbar_arrive(BAR(kBarEmpty + slot));
                     if (++slot == (uint32_t)kRing) { slot = 0; full_par ^= 1u; }
                     if (++in_round == per_round) { in_round = 0; ++round; active = round < work.rounds && t < work.round_size(round); }
-                    continue;
+                    continue;                                       // (an idle round keeps `stage` at 0: it is only read while active)
                 }
                 if (ok && s_in == 0) ok = mbar_wait(bar_ready, ready_par, abort_flag);
                 if (ok && !first) ok = mbar_wait(bar_free, free_par, abort_flag);
@@ -430,10 +443,26 @@ encode_tensor_kernel(const Params p)
                     mma_commit(BAR(kBarEmpty + slot));
                 }
                 __syncwarp();
+                if (p.defer_stats && stage >= 1u && s_in >= 1u && s_in <= 4u) {
+                    const int rl = t * 128 + (int)(s_in - 1u) * 32 + lane;
+                    const uint32_t fl = flags_s[rl];
+                    if (fl & 1u) {
+                        const size_t bin = (size_t)(stage - 1u) * s.K + codes_s[rl * 16 + (int)(stage - 1u)];
+                        atomicAdd(p.stat_cnt + bin, 1u);
+                        if (!(fl & 2u)) {
+                            float4 *m = reinterpret_cast<float4 *>(p.stat_sum + bin * 32);
+#pragma unroll
+                            for (int q4 = 0; q4 < 8; ++q4)
+                                atomicAdd(m + q4, make_float4(zp[(4 * q4) * kRowsPerPass + rl], zp[(4 * q4 + 1) * kRowsPerPass + rl],
+                                                              zp[(4 * q4 + 2) * kRowsPerPass + rl], zp[(4 * q4 + 3) * kRowsPerPass + rl]));
+                        }
+                    }
+                    __syncwarp();
+                }
                 free_par ^= 1u;
                 if (++slot == (uint32_t)kRing) { slot = 0; full_par ^= 1u; }
-                if (++s_in == (uint32_t)S) { s_in = 0; ready_par ^= 1u; }
-                if (++in_round == per_round) { in_round = 0; ++round; active = round < work.rounds && t < work.round_size(round); }
+                if (++s_in == (uint32_t)S) { s_in = 0; ready_par ^= 1u; ++stage; }
+                if (++in_round == per_round) { in_round = 0; stage = 0; ++round; active = round < work.rounds && t < work.round_size(round); }
             }
         }
     } else {
@@ -523,6 +552,7 @@ encode_tensor_kernel(const Params p)
             }
             // (raw rows are stage inputs already: taken as they are, no deviation stored)
             const bool deg = s.raw ? !valid : (deviation_is_degenerate(dev) || !valid);
+            if (p.defer_stats) smem[kOffFlags + rloc] = (uint8_t)((valid ? 1 : 0) | (deg ? 2 : 0));
 #pragma unroll
             for (int i = 0; i < 32; ++i) z[i] = deg ? 0.0f : (s.raw ? z[i] : z[i] / dev);
             if (valid && g == 0 && !s.raw) {
@@ -709,8 +739,9 @@ encode_tensor_kernel(const Params p)
                     }
                 }
                 if (deg) bj = 0;
-                if (p.stat_sum && valid) {
+                if (p.stat_sum && valid && !(p.defer_stats && r < s.R - 1)) {
                     // EMA statistics (Section 3): this row's stage input joins the bin of its code
+                    // (all stages but the last are the issuer warps' when deferred)
                     const size_t bin = (size_t)r * s.K + bj;
                     atomicAdd(p.stat_cnt + bin, 1u);
                     if (!deg) {
@@ -801,6 +832,13 @@ bool encode_tensor_supported(const Shape &s)
     return s.gd == 32 && s.G <= 32 && (s.G & (s.G - 1)) == 0 && slots_per_stage(s.K) * 4 <= 65535;
 }
 
+// Stages 0 .. this - 1 of the fused statistics hold the sums of what those stages LEFT (their bins' inputs
+// minus count * codeword): the caller adds count * codeword (launch_stats_finish).
+int encode_tensor_deferred_stages(const Shape &s)
+{
+    return encode_tensor_supported(s) && slots_per_stage(s.K) >= kDeferMinSlots && s.R > 1 ? s.R - 1 : 0;
+}
+
 int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t stride, const float *cb,
                          const void *prepared, void *codes, uint16_t *std16, rvq_status *st,
                          cudaStream_t stream, uint32_t *stat_cnt, float *stat_sum, float *energy,
@@ -817,7 +855,8 @@ int launch_encode_tensor(const Shape &s, const void *x, int64_t n, int64_t strid
     if (cudaFuncSetAttribute(encode_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
         return RVQ_ERR_LAUNCH;
     Params p{s, x, n, stride, cb, reinterpret_cast<const uint8_t *>(prepared), codes, std16, st, (int)tiles, stat_cnt, stat_sum,
-             energy, wait_limit ? wait_limit : kWaitLimit, drop_last_chain};
+             energy, wait_limit ? wait_limit : kWaitLimit, drop_last_chain,
+             stat_sum != nullptr && encode_tensor_deferred_stages(s) > 0 ? 1 : 0};
     const int64_t groups = (tiles + kTiles - 1) / kTiles;
     const int grid = (int)(groups < sms ? groups : sms);
     encode_tensor_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);

@@ -34,6 +34,10 @@
 //   - The float32 residual lives in registers between stages and is parked in
 //     shared memory during a stage's sweep; x is read once and only codes and
 //     the half-precision deviation are written.
+//   - With the EMA statistics asked for (Section 3), every stage's rows join the bins of their codes:
+//     the stage's output, parked for the next sweep, is added by the tile's MMA issuer warp between
+//     two chains of that sweep (count x codeword is added back by the caller's finishing kernel); the
+//     last stage's input is added by the epilogue warps.
 // TMEM columns of tile t: scores [160 t, 160 t + 128), A operand
 // [160 t + 128, 160 t + 160) (16 columns of head, 16 of remainder).
 // Every wait is bounded; a wait that gives up sets status->wait_timeouts and
